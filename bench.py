@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the SparQ decode hot path on B200.
+
+A step is one pass of the whole path over one batch: ``sparq_cache_append`` of one new token per
+sequence followed by ``sparq_decode`` of one query per (sequence, head).  Workload: the batched
+Llama-2-7B-shaped case (B=64, 32 heads, d_h=128, S=4096, r=32, k=128, fp16 cache; the shape of
+the paper's GPU microbenchmark table), synthetic and seeded.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl b200|reference]
+
+N > 1 is launched by torchrun, one rank per GPU; the (batch, head) units are independent, so each
+rank runs its own batch of the same shape (weak scaling) and there is no data-path collective.
+Rank 0 prints one JSON line.  ``--impl reference`` times the float64 CPU oracle on a bounded
+sample of the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparq_decode tokens*heads/s (us/step, HBM GB/s on compulsory bytes, speed-up vs dense_decode alongside)"
+UNIT = "tokens*heads/s"
+WORKLOAD = "c2"
+PERIOD = 64          # steps between rewinds of seq_lens (the cache would otherwise fill up)
+POOL = 16            # distinct (q, k_new, v_new) sets rotated through the steps
+L2_BYTES = 126e6
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
+# from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def compulsory_bytes_per_unit(n: float, r: int, k: int, d: int) -> float:
+    """fp16 bytes one (batch, query head) must move: r rows of Kt over n positions, k rows each
+    of K and V, plus q, v_bar and the output (Eq. (11) x 2 bytes, without the append term)."""
+    return 2.0 * n * r + 4.0 * k * d + 6.0 * d
+
+
+def dense_bytes(B, Hq, Hkv, n, d):
+    return B * Hkv * 4.0 * n * d + B * Hq * 4.0 * d
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
+
+    def summary(self) -> dict:
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for row in self.rows:
+            if len(row) < 7:
+                continue
+            try:
+                sm.append(float(row[0]))
+                smax.append(float(row[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, row[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _sample_units(case, n_units, seed=0):
+    """A bounded, seeded sample of (b, h) units with their KV heads copied to the host as fp16 numpy:
+    q [U,1,d], K,V [U,1,S_max,d], seq [U] -- each unit becomes a batch element of a 1-head problem."""
+    import numpy as np
+    import torch
+    g = torch.Generator().manual_seed(seed)
+    U = min(n_units, case.B * case.Hq)
+    flat = torch.randperm(case.B * case.Hq, generator=g)[:U]
+    bs, hs = flat // case.Hq, flat % case.Hq
+    grp = case.Hq // case.Hkv
+    qdev = case.q_steps.device
+    q = case.q_steps[-1][bs.to(qdev), hs.to(qdev)].unsqueeze(1).cpu().numpy()
+    K = torch.stack([case.K[b, h // grp] for b, h in zip(bs.tolist(), hs.tolist())]).unsqueeze(1).cpu().numpy()
+    V = torch.stack([case.V[b, h // grp] for b, h in zip(bs.tolist(), hs.tolist())]).unsqueeze(1).cpu().numpy()
+    seq = (case.seq_lens.cpu() + case.n_steps)[bs].numpy().astype(np.int32)
+    return q, K, V, seq
+
+
+def time_oracle(case, n_units, reps=1):
+    """The C float64 oracle, as it stands, on a sample of units with every host core OpenMP gives it."""
+    from oracle import c_oracle
+    q, K, V, seq = _sample_units(case, n_units)
+    cores = c_oracle.max_threads()
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        c_oracle.sparq_decode(q, K, V, seq, case.r, case.k)
+        times.append(time.perf_counter() - t0)
+    return len(seq), cores, times
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, same metric and workload, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from paper_2312_04985_b200 import synth
+    n_units = 64
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    case = synth.make_case(WORKLOAD, device=dev, B=2)           # the sample only needs a few sequences' caches
+    from oracle import c_oracle
+    c_oracle.build()
+    U, cores, _ = time_oracle(case, n_units, reps=max(1, min(args.warmup, 1)))
+    _, _, times = time_oracle(case, n_units, reps=max(1, min(args.steps, 5)))
+    t = sum(times) / len(times)
+    value = U / t
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": len(times), "warmup": 1, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "c2: B=64 Hq=Hkv=32 d=128 S=4096 r=32 k=128 fp16 cache",
+                       "sample": "%d of 2048 (batch, head) units per step" % U},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": "%d (b,h) units of c2 per step, C float64 oracle, OpenMP over units" % U},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_b200(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2312_04985_b200 import sparq, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SparQ path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    sparq.lib()                                                  # fail loudly if the library is missing
+
+    # ---------------------------------------------------------------- workload (per rank, own seed)
+    case = synth.make_case(WORKLOAD, device=str(dev), seed=synth.SPECS[WORKLOAD]["seed"] + 1000 * rank,
+                           B=args.batch)
+    B, Hq, Hkv, d, S_max, r, k = case.B, case.Hq, case.Hkv, case.d, case.S_max, case.r, case.k
+    pool = synth.make_step_pool(case, POOL)
+    K, V = case.K, case.V
+    Kt = torch.zeros(B, Hkv, d, S_max, dtype=torch.float16, device=dev)
+    vsum = torch.zeros(B, Hkv, d, dtype=torch.float32, device=dev)
+    vbar = torch.zeros(B, Hkv, d, dtype=torch.float16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    period = min(PERIOD, S_max - 8)
+    seq_start = torch.full((B,), S_max - period, dtype=torch.int32, device=dev)
+    seq_full = torch.full((B,), S_max, dtype=torch.int32, device=dev)
+    seq_lens = seq_start.clone()
+    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)    # state at the start of a period
+    vsum_start = vsum.clone()
+    out = torch.empty(B, Hq, d, dtype=torch.float16, device=dev)
+    torch.cuda.synchronize()
+
+    def rewind():
+        # start a period: lengths (and the running value sum) back to S - period; stream-ordered
+        # device copies of B and B*Hkv*d elements, inside the timed region
+        seq_lens.copy_(seq_start)
+        vsum.copy_(vsum_start)
+
+    def step(i, ev=None):
+        if i % period == 0:
+            rewind()
+        j = i % POOL
+        sparq.sparq_cache_append(pool["k_new"][j], pool["v_new"][j], K, Kt, V, vsum, vbar, seq_lens, status)
+        if ev is not None:
+            ev[0].record()
+        sparq.sparq_decode(pool["q"][j], K, Kt, V, vbar, seq_lens, r, k, out, status=status)
+        if ev is not None:
+            ev[1].record()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---------------------------------------------------------------- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        time.sleep(0.25)
+        barrier()
+        t_beg.record()
+        for i in range(args.steps):
+            step(i, evs[i])
+        t_end.record()
+        barrier()
+        # keep the GPU in the same loop a little longer so the 200 ms sampler sees it under load
+        t_load = time.perf_counter()
+        i = 0
+        while time.perf_counter() - t_load < 1.0:
+            step(i)
+            i += 1
+            if i % 32 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+    total_ms = max_over_ranks(t_beg.elapsed_time(t_end))
+    decode_ms = [a.elapsed_time(b) for a, b in evs]
+    decode_us = max_over_ranks(1e3 * sum(decode_ms) / len(decode_ms))
+    if int(status.item()) != 0:
+        raise SystemExit("device status %s" % sparq.status_string(int(status.item())))
+    us_per_step = 1e3 * total_ms / args.steps
+    units = B * Hq * world
+    value = units / (us_per_step * 1e-6)
+    n_mean = sum(S_max - period + (i % period) + 1 for i in range(args.steps)) / args.steps
+    bytes_launch = B * Hq * compulsory_bytes_per_unit(n_mean, r, k, d)
+    achieved = bytes_launch / (decode_us * 1e-6) / 1e9
+    peak, peak_kind = _peaks()
+
+    # ---------------------------------------------------------------- dense_decode on the same cache
+    ws = torch.empty(max(sparq.dense_workspace_bytes(B, Hq, Hkv, d, S_max), 4), dtype=torch.uint8, device=dev)
+    seq_lens.copy_(seq_full)
+    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)    # whole cache valid: full-length comparison
+    dn_steps = max(3, min(args.steps, 30))
+    for i in range(3):
+        sparq.dense_decode(pool["q"][i % POOL], K, V, seq_lens, out, workspace=ws, status=status)
+    barrier()
+    t_beg.record()
+    for i in range(dn_steps):
+        sparq.dense_decode(pool["q"][i % POOL], K, V, seq_lens, out, workspace=ws, status=status)
+    t_end.record()
+    barrier()
+    dense_us = max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / dn_steps)
+    # sparq_decode alone at the same full length, for the speed-up figure
+    for i in range(3):
+        sparq.sparq_decode(pool["q"][i % POOL], K, Kt, V, vbar, seq_lens, r, k, out, status=status)
+    barrier()
+    t_beg.record()
+    for i in range(dn_steps):
+        sparq.sparq_decode(pool["q"][i % POOL], K, Kt, V, vbar, seq_lens, r, k, out, status=status)
+    t_end.record()
+    barrier()
+    sparq_full_us = max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / dn_steps)
+
+    # ---------------------------------------------------------------- end to end from host buffers
+    staging = torch.empty(sparq.sparq_step_host_staging_bytes(B, Hq, Hkv, d), dtype=torch.uint8, device=dev)
+    hq = [pool["q"][j].cpu().pin_memory() for j in range(POOL)]
+    hk = [pool["k_new"][j].cpu().pin_memory() for j in range(POOL)]
+    hv = [pool["v_new"][j].cpu().pin_memory() for j in range(POOL)]
+    hout = torch.empty(B, Hq, d, dtype=torch.float16).pin_memory()
+
+    def host_step(i):
+        if i % period == 0:
+            rewind()
+        j = i % POOL
+        sparq.sparq_step_host(hq[j], hk[j], hv[j], K, Kt, V, vsum, vbar, seq_lens, r, k, hout, staging, status)
+
+    seq_lens.copy_(seq_start)
+    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)
+    vsum_start.copy_(vsum)
+    for i in range(max(3, args.warmup // 2)):
+        host_step(i)
+    barrier()
+    e2e_steps = args.steps
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        host_step(i)
+    torch.cuda.synchronize()
+    e2e_s = max_over_ranks(time.perf_counter() - t0)
+    e2e_value = units * e2e_steps / e2e_s
+    h2d = (B * Hq * d + 2 * B * Hkv * d) * 2
+    d2h = B * Hq * d * 2
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---------------------------------------------------------------- CPU baseline: the oracle on the host cores
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import c_oracle
+        c_oracle.build()
+        U, cores, times = time_oracle(case, 128, reps=1)        # warm-up (page-in, OpenMP pool)
+        target_units = int(min(B * Hq, max(128, 15.0 * U / max(times[0], 1e-3))))   # about 15 s of CPU work
+        U, cores, times = time_oracle(case, target_units, reps=1)
+        cpu = {"value": U / times[0], "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "%d of %d (b,h) units of c2 (seeded sample), one pass, C float64 oracle with OpenMP "
+                         "over units, %.1f s" % (U, B * Hq, times[0])}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": us_per_step / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64 approximate-score accumulation over fp16 cache; f32 softmax and value accumulation",
+        "data": "synthetic",
+        "config": {"workload": "c2: B=%d Hq=%d Hkv=%d d=%d S=%d r=%d k=%d fp16 cache, per GPU" % (B, Hq, Hkv, d, S_max, r, k),
+                   "step": "sparq_cache_append + sparq_decode; seq_lens rewound to S-%d every %d steps" % (period, period),
+                   "l2": "inputs larger than L2 (cache %.2f GB vs 126 MB L2); q/k/v rotate over %d sets"
+                         % (3 * K.numel() * 2 / 1e9, POOL),
+                   "parallelism": "independent batches per GPU, no collective"},
+        "us_per_step": us_per_step, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
+        "dense_decode_us": dense_us, "speedup_vs_dense": dense_us / sparq_full_us,
+        "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, S_max, d) / (dense_us * 1e-6) / 1e9,
+        "hbm_gbs_compulsory": achieved, "frac_of_8tbs": achieved / 8000.0,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "sparq_decode_kernel",
+                     "algorithmic_bytes_per_launch": bytes_launch, "peak_kind": peak_kind + " (copy bandwidth)"},
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "us_per_step": 1e6 * e2e_s / e2e_steps, "api": "sparq_step_host (pinned host q, k_new, v_new -> host out)"},
+        "gpu_launches": 3 * args.steps,
+        "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--batch", type=int, default=None, help="override B (profiling on a small case only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_b200(args)
+
+
+if __name__ == "__main__":
+    main()

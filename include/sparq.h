@@ -1,0 +1,144 @@
+/*
+ * sparq.h -- C ABI of the B200 (sm_100a) SparQ decode-attention library.
+ *
+ * SparQ Attention (arXiv 2312.04985) replaces the dense single-token decode attention
+ *     y = softmax(q K^T / sqrt(d_h)) V                                   (Eq. (2))
+ * by three steps per query head (Section 4):
+ *   Step 1  i1 = the r largest components of |q|; approximate scores
+ *           s_hat = softmax(q[i1] K[:, i1]^T / tau),  tau = sqrt(d_h ||q[i1]||_1 / ||q||_1)
+ *                                                                         (Eqs. (7), (9))
+ *   Step 2  i2 = the k positions with the largest s_hat; exact attention over them
+ *           y3 = softmax(q K[i2]^T / sqrt(d_h)) V[i2]                      (Eq. (8))
+ *   Step 3  alpha = sum of s_hat over i2;  y = alpha y3 + (1 - alpha) v_bar (Eq. (10))
+ * with v_bar the running mean of the cached value vectors (Section 3, "Mean value
+ * reallocation").  K is stored twice (Section 6): K, position-major [S, d_h], for the row
+ * gather of Step 2, and Kt, component-major [d_h, S], for the component gather of Step 1.
+ *
+ * Conventions common to every call
+ *   - fp16 tensors are passed as `const sparq_half*` (IEEE binary16 bit patterns).
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller.
+ *     The library allocates no device memory and keeps no pointer after the call returns.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and return without synchronising, except the *_host entry points.
+ *   - Layouts (row-major, innermost last):
+ *         q, out        [B, Hq, d]
+ *         K, V          [B, Hkv, S_max, d]
+ *         Kt            [B, Hkv, d, S_max]
+ *         vsum (fp32), vbar (fp16), k_new, v_new   [B, Hkv, d]
+ *         seq_lens (int32)   [B]     number of valid positions of sequence b
+ *     Query head h reads KV head h / (Hq / Hkv): consecutive query heads share a KV head
+ *     (Section 4, "Grouped query attention").  Each query head selects its own i1 and i2.
+ *   - Supported shapes: d == 128; Hq a multiple of Hkv; S_max a multiple of 8 (rows of Kt
+ *     are then 16-byte aligned); 1 <= r <= d; 0 <= k <= SPARQ_K_MAX.
+ *   - Return value: SPARQ_OK, or a SPARQ_ERR_* code for anything the host can see; in that
+ *     case nothing was launched.  Conditions only the device can see (a bad seq_lens[b], an
+ *     append into a full cache) never trap: the kernel raises `*status` (device int32,
+ *     may be NULL) to a SPARQ_DEV_* code with atomicMax, writes a defined result for that
+ *     sequence (zeros / no write) and carries on.  The caller zeroes `*status` and reads it
+ *     whenever it wants to check.
+ *   - Non-finite cache values are not supported (no fault; the result is unspecified).
+ */
+#ifndef SPARQ_H
+#define SPARQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t sparq_half;
+
+#define SPARQ_K_MAX 1024
+#define SPARQ_HEAD_DIM 128
+
+enum {
+    SPARQ_OK = 0,
+    SPARQ_ERR_NULL_POINTER = 1,  /* a required pointer is NULL                                   */
+    SPARQ_ERR_BAD_SHAPE = 2,     /* B, Hq, Hkv, d or S_max outside the supported shapes          */
+    SPARQ_ERR_BAD_RK = 3,        /* r or k out of range                                          */
+    SPARQ_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than *_workspace_bytes()           */
+    SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds what the kernels' on-chip score buffer holds   */
+    SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
+    SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */
+    SPARQ_DEV_CACHE_FULL = 17    /* device: append with seq_lens[b] == S_max; nothing written    */
+};
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* sparq_status_string(int code);
+
+/* Largest S_max sparq_decode accepts on the current device (limited by shared memory). */
+int sparq_max_seq_len(void);
+
+/*
+ * sparq_cache_build -- derive the SparQ-specific cache state from a prefilled K, V:
+ * Kt[b,h,:,t] = K[b,h,t,:] for t < seq_lens[b] (Section 6, "store K twice"), the fp32
+ * running sum vsum = sum_{t<n} V[b,h,t,:] and vbar = fp16(vsum / n) (Section 3, v_bar).
+ * Positions t >= seq_lens[b] of Kt are left untouched.  seq_lens[b] == 0 gives vsum = vbar = 0.
+ */
+int sparq_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                      sparq_half* Kt, float* vsum, sparq_half* vbar,
+                      int B, int Hkv, int d, int S_max, int32_t* status, void* stream);
+
+/*
+ * sparq_cache_append -- one generation step's cache update (Section 3, text around Eq. (3);
+ * Appendix "Storing K twice").  For every sequence b, with n = seq_lens[b] read at entry, every
+ * KV head writes k_new to K[b,h,n,:] and to Kt[b,h,:,n], v_new to V[b,h,n,:], adds v_new to
+ * vsum and refreshes vbar = fp16(vsum / (n + 1)); then seq_lens[b] becomes n + 1.  A decode
+ * enqueued after the append on the same stream attends to the new token.
+ * n == S_max: nothing is written for b, seq_lens[b] is unchanged, *status = SPARQ_DEV_CACHE_FULL.
+ */
+int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
+                       sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
+                       int32_t* seq_lens, int B, int Hkv, int d, int S_max, int32_t* status, void* stream);
+
+/*
+ * sparq_decode -- the SparQ attention step (Section 4, Steps 1-3) for every (b, query head).
+ * With n = seq_lens[b] and k_eff = min(k, n):
+ *   i1 (r components, ties in |q| to the smaller index), tau (Eq. (9); an all-zero q uses tau = 1),
+ *   l_hat[t] = sum_{j in i1} q_j K[t,j] / tau for t < n, accumulated in fp64 (Eq. (7)),
+ *   i2 = the k_eff largest l_hat (ties to the smaller position), alpha = sum_{t in i2} s_hat[t],
+ *   y3 = softmax(q K[i2]^T / sqrt(d)) V[i2] in fp32 (Eq. (8)), out = alpha y3 + (1-alpha) vbar
+ *   rounded to fp16 (Eq. (10)).  k == 0 gives out = vbar.
+ * Optional outputs (each may be NULL): idx_r [B,Hq,r] int32 = i1 ascending; idx_k [B,Hq,k]
+ * int32 = i2 ascending, unused tail -1; alpha [B,Hq] fp32.
+ * workspace: reserved for plans that need scratch; sparq_workspace_bytes() says how much
+ * (0 for the current single-kernel plan, in which case workspace may be NULL).
+ */
+int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                 const sparq_half* vbar, const int32_t* seq_lens,
+                 int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                 sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k);
+
+/*
+ * dense_decode -- dense decode attention, Eq. (2), over the n = seq_lens[b] valid positions:
+ * the comparison kernel for the speed-up figure (Section 6.1, "Dense" baseline).  One pass
+ * over K and V per KV head serves all Hq/Hkv query heads of its group.  The sequence is split
+ * across thread blocks; partial softmax states go through `workspace`
+ * (dense_workspace_bytes(); contents undefined afterwards).
+ */
+int dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                 int B, int Hq, int Hkv, int d, int S_max, sparq_half* out,
+                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
+
+/*
+ * sparq_step_host -- one whole generation step driven from HOST buffers: copies q_host
+ * [B,Hq,d], k_new_host and v_new_host [B,Hkv,d] (fp16, ideally pinned) to the device, runs
+ * sparq_cache_append then sparq_decode on `stream`, copies the result to out_host [B,Hq,d]
+ * and waits for the stream.  The cache (K, Kt, V, vsum, vbar, seq_lens) stays resident on the
+ * device.  staging: device scratch of at least sparq_step_host_staging_bytes() bytes.
+ */
+int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, const sparq_half* v_new_host,
+                    sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
+                    int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                    sparq_half* out_host, void* staging, size_t staging_bytes, int32_t* status, void* stream);
+size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARQ_H */

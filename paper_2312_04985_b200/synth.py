@@ -176,3 +176,27 @@ def make_case(name: str, *, device: str = "cpu", backend: Optional[str] = None, 
     v_steps = torch.gather(V.unsqueeze(0).expand(steps, -1, -1, -1, -1), 3, gather_idx).squeeze(3).contiguous()
     return Case(name=name, B=B_, Hq=Hq_, Hkv=Hkv_, d=d, S_max=S_max, r=spec["r"], k=spec["k"], seed=spec["seed"],
                 n_steps=steps, K=K, V=V, seq_lens=seq0, q_steps=q, k_steps=k_steps, v_steps=v_steps)
+
+
+def make_step_pool(case: Case, n: int, *, seed: int = 1000) -> dict:
+    """Extra per-step inputs for timing loops: ``n`` fresh queries drawn by the case's query
+    recipe (pool[0] is the case's own last-step query) and ``n`` fresh N(0,1) tokens to append.
+    Returns q [n,B,Hq,d], k_new, v_new [n,B,Hkv,d] (fp16, on the case's device)."""
+    spec = SPECS[case.name]
+    dev = case.K.device
+    rng = _Rng(seed + case.seed, "torch", str(dev))
+    q = rng.normal(n, case.B, case.Hq, case.d)
+    if spec["qheavy"]:
+        nh, scale = spec["qheavy"]
+        dims = rng.distinct(n * case.B * case.Hq, case.d, nh).view(n, case.B, case.Hq, nh)
+        mult = torch.ones_like(q)
+        mult.scatter_(3, dims, scale)
+        q = q * mult
+    q = q.to(torch.float16)
+    q[0] = case.q_steps[-1]
+    k_new = rng.normal(n, case.B, case.Hkv, case.d)
+    if spec["student"]:
+        chi = rng.normal(n, case.B, case.Hkv, 3).square().sum(-1, keepdim=True) / 3.0
+        k_new = k_new / chi.sqrt()
+    v_new = rng.normal(n, case.B, case.Hkv, case.d)
+    return dict(q=q, k_new=k_new.to(torch.float16), v_new=v_new.to(torch.float16))

@@ -1,0 +1,240 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 oracle on the
+same seeded fp16 inputs.  Acceptance rule: index sets bit-exact unless the oracle's boundary gap
+is below 1e-6 relative; outputs within 2e-3 max-abs and 1e-3 relative L2."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import c_oracle, sparq_oracle as O
+from paper_2312_04985_b200 import sparq, synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _dense_check(case, cache, q, what):
+    got = cache.dense(q)
+    seq = cache.seq_lens.cpu().numpy()
+    want = c_oracle.dense_decode(q.numpy(), case.K.numpy(), case.V.numpy(), seq)
+    H.check_out(got.reshape(want.shape), want, what + " dense")
+
+
+# ------------------------------------------------------------------ the paper-shaped workloads
+def test_c0_tiny_single_step_against_numpy_oracle():
+    c = synth.make_case("c0")
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens)
+    cache.append(c.k_steps[0], c.v_steps[0])
+    gpu = cache.decode(c.q_steps[0], c.r, c.k)
+    ora = O.sparq_decode(c.q_steps[0].numpy(), c.K.numpy(), c.V.numpy(), [512], c.r, c.k, fast=False)
+    np.testing.assert_array_equal(gpu["i1"], ora["i1"])
+    np.testing.assert_array_equal(gpu["i2"], ora["i2"])
+    assert abs(gpu["alpha"][0, 0] - ora["alpha"][0, 0]) <= H.ALPHA_TOL
+    H.check_out(gpu["out"], ora["out"], "c0")
+    # the running mean after the append against the from-scratch float64 mean
+    vb = O.mean_value(c.V[0, 0].numpy().astype(np.float64), 512)
+    np.testing.assert_allclose(cache.vbar[0, 0].cpu().numpy().astype(np.float64), vb, atol=2e-4)
+    np.testing.assert_allclose(cache.vsum[0, 0].cpu().numpy().astype(np.float64), vb * 512, rtol=0, atol=2e-3)
+    cache.check_status(0)
+    _dense_check(c, cache, c.q_steps[0], "c0")
+
+
+def test_c1_llama2_batch1_all_heads():
+    c = synth.make_case("c1")
+    waived, total = H.run_case_all_heads(c, "c1")
+    assert total == 32 and waived <= 1
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("c2", dict(B=3)),
+    ("c3", dict(B=2)),
+    ("c4", dict(B=2, n_steps=3)),
+    ("c4", dict(B=3, n_steps=2, ragged=(1000, 3000), Hq=8, Hkv=2)),
+])
+def test_shrunk_batch_all_heads(name, kw):
+    c = synth.make_case(name, device="cuda", **kw)
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    waived, total = H.run_case_all_heads(c, name)
+    assert waived <= max(1, total // 200)
+
+
+def test_dense_decode_on_workloads():
+    for name, kw in (("c1", {}), ("c3", dict(B=2, S=5000, backend="numpy")),
+                     ("c4", dict(B=3, n_steps=1, ragged=(700, 2500), backend="numpy"))):
+        c = synth.make_case(name, **kw)
+        cache = H.DeviceCache(c.K, c.V, c.seq_lens + c.n_steps, poison=True)
+        _dense_check(c, cache, c.q_steps[-1], name)
+        cache.check_status(0)
+
+
+# ------------------------------------------------------------------ edge cases
+def _small(B=2, Hq=4, Hkv=2, S=96, seed=11, n=None):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(B, Hq, 128, generator=g)
+    q[..., :5] *= 6
+    K = torch.randn(B, Hkv, S, 128, generator=g).half()
+    V = torch.randn(B, Hkv, S, 128, generator=g).half()
+    seq = torch.tensor(n if n is not None else [S] * B, dtype=torch.int32)
+    return q.half(), K, V, seq
+
+
+def _compare_all(q, K, V, seq, r, k, what):
+    cache = H.DeviceCache(K, V, seq)
+    gpu = H.flat(cache.decode(q, r, k))
+    B, Hq, _ = q.shape
+    g = Hq // K.shape[1]
+    Knp, Vnp, qn = K.numpy(), V.numpy(), q.numpy()
+    ora = c_oracle.sparq_decode(qn, Knp, Vnp, seq.numpy(), r, k)
+    waived = H.compare_units(gpu, ora, qn.reshape(B * Hq, -1), lambda u: Knp[u // Hq, (u % Hq) // g],
+                             lambda u: Vnp[u // Hq, (u % Hq) // g], np.repeat(seq.numpy(), Hq), r, k, what)
+    cache.check_status(0)
+    return cache, gpu, ora, waived
+
+
+@pytest.mark.parametrize("n,r,k", [
+    ([1, 1], 4, 4),          # single position
+    ([7, 96], 16, 32),       # n < 8, n < k: k clipped to n
+    ([61, 33], 128, 8),      # r = d_h; ragged tails inside a 16-byte vector
+    ([96, 50], 1, 1),        # smallest r and k
+    ([96, 96], 17, 96),      # r not a multiple of the row batch; k = n
+    ([95, 90], 128, 1024),   # r = d_h and k >= n: dense attention
+])
+def test_edge_sizes(n, r, k):
+    q, K, V, seq = _small(n=n)
+    cache, gpu, ora, waived = _compare_all(q, K, V, seq, r, k, "edge n=%s r=%d k=%d" % (n, r, k))
+    assert waived == 0
+    if r == 128 and k >= max(n):
+        dn = cache.dense(q)
+        H.check_out(gpu["out"], dn.reshape(gpu["out"].shape), "sparq(r=d,k=n) vs dense_decode")
+        np.testing.assert_allclose(gpu["alpha"], 1.0, atol=H.ALPHA_TOL)
+
+
+def test_k_zero_returns_vbar():
+    q, K, V, seq = _small(n=[40, 96])
+    cache = H.DeviceCache(K, V, seq)
+    gpu = cache.decode(q, 8, 0)
+    vb = cache.vbar.cpu().numpy().astype(np.float64)
+    np.testing.assert_array_equal(gpu["out"], np.repeat(vb, 2, axis=1))
+    np.testing.assert_array_equal(gpu["alpha"], 0.0)
+    want = np.stack([np.stack([V[b, h, : seq[b]].double().mean(0).numpy() for h in range(2)]) for b in range(2)])
+    np.testing.assert_allclose(vb, want, atol=2e-4)
+
+
+def test_exact_ties_resolve_to_lower_index():
+    q, K, V, seq = _small(B=1, Hq=2, Hkv=1, S=64)
+    # all-zero query: every |q_j| ties, tau := 1, all logits 0 -> i1 = first r, i2 = first k
+    q[0, 0] = 0
+    # duplicated key rows: positions 2t and 2t+1 score identically
+    K[0, 0, 1::2] = K[0, 0, 0::2]
+    cache, gpu, ora, waived = _compare_all(q, K, V, seq, 8, 9, "ties")
+    assert gpu["i1"][0].tolist() == list(range(8))
+    assert gpu["i2"][0].tolist() == list(range(9))
+    assert abs(gpu["alpha"][0] - 9 / 64) < 1e-6
+    assert ora["gap_k"][1] == 0.0 or gpu["i2"][1].tolist() == ora["i2"][1].tolist()
+    # +0 and -0 magnitudes and repeated |q| values tie exactly in fp16
+    q2 = torch.zeros(1, 1, 128, dtype=torch.float16)
+    q2[0, 0, [3, 9, 40, 41, 100]] = torch.tensor([2.0, -2.0, 2.0, -0.0, 2.0], dtype=torch.float16)
+    cache2, gpu2, ora2, _ = _compare_all(q2, K[:, :1], V[:, :1], seq, 3, 5, "q ties")
+    assert gpu2["i1"][0].tolist() == [3, 9, 40]
+
+
+def test_fp32_ties_are_decided_in_fp64():
+    """Approximate logits that agree to fp32 rounding but differ in fp64 (and some that are
+    exactly equal) at the k-th place: the selection must follow the float64 order."""
+    S, r = 200, 2
+    rng = np.random.default_rng(5)
+    q = torch.zeros(1, 1, 128, dtype=torch.float16)
+    q[0, 0, 10] = 1024.0
+    q[0, 0, 77] = 2.0 ** -14
+    K = torch.zeros(1, 1, S, 128, dtype=torch.float16)
+    K[0, 0, :, 10] = 1.0
+    K[0, 0, :, 77] = torch.from_numpy(rng.integers(1, 40, S) / 128.0).half()   # < half an fp32 ulp of 1024
+    K[0, 0, 5, 10] = 1.5                                                       # one clear winner
+    K[0, 0, 6, 10] = 0.5                                                       # one clear loser
+    V = torch.from_numpy(rng.standard_normal((1, 1, S, 128))).half()
+    seq = torch.tensor([S], dtype=torch.int32)
+    for k in (1, 2, 17, 64, 199):
+        cache, gpu, ora, waived = _compare_all(q, K, V, seq, r, k, "fp64 ties k=%d" % k)
+        assert np.array_equal(gpu["i2"][0], ora["i2"][0])
+    lh = 1024.0 * K[0, 0, :, 10].double() + 2.0 ** -14 * K[0, 0, :, 77].double()
+    assert len(set(lh.float().tolist())) == 3 and len(set(lh.tolist())) > 20   # the case is what it claims
+
+
+def test_repeat_launches_are_bitwise_identical():
+    c = synth.make_case("c1", Hq=8, Hkv=8)
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
+    a = cache.decode(c.q_steps[0], c.r, c.k)
+    b = cache.decode(c.q_steps[0], c.r, c.k)
+    for key in a:
+        np.testing.assert_array_equal(a[key], b[key])
+
+
+def test_permuting_positions_permutes_the_selection():
+    q, K, V, seq = _small(B=1, Hq=2, Hkv=1, S=300)
+    cache = H.DeviceCache(K, V, seq)
+    base = cache.decode(q, 16, 24)
+    perm = torch.randperm(300, generator=torch.Generator().manual_seed(3))
+    cache2 = H.DeviceCache(K[:, :, perm], V[:, :, perm], seq)
+    res = cache2.decode(q, 16, 24)
+    for h in range(2):
+        assert sorted(perm[res["i2"][0, h]].tolist()) == base["i2"][0, h].tolist()
+    np.testing.assert_allclose(res["out"], base["out"], atol=2e-3)
+
+
+# ------------------------------------------------------------------ error behaviour on the device
+def test_bad_seq_len_sets_status_and_zero_row():
+    q, K, V, seq = _small(B=3, n=[96, 0, 50])
+    cache = H.DeviceCache(K, V, torch.tensor([96, 96, 50], dtype=torch.int32))
+    cache.seq_lens.copy_(torch.tensor([96, 0, 50], dtype=torch.int32))
+    gpu = cache.decode(q, 8, 8)
+    cache.check_status(sparq.DEV_BAD_SEQ_LEN)
+    assert (gpu["out"][1] == 0).all() and (gpu["i2"][1] == -1).all() and (gpu["i1"][1] == -1).all()
+    assert np.isfinite(gpu["out"]).all() and (gpu["out"][0] != 0).any() and (gpu["out"][2] != 0).any()
+    cache.status.zero_()
+    cache.seq_lens.copy_(torch.tensor([96, 97, 50], dtype=torch.int32))     # beyond capacity
+    dn = cache.dense(q)
+    cache.check_status(sparq.DEV_BAD_SEQ_LEN)
+    assert (dn[1] == 0).all() and np.isfinite(dn).all()
+
+
+def test_append_into_full_cache_is_refused():
+    q, K, V, seq = _small(B=2, n=[96, 95])
+    cache = H.DeviceCache(K, V, seq, poison=False)
+    K0 = cache.K.clone()
+    kn = torch.ones(2, 2, 128, dtype=torch.float16)
+    cache.append(kn, kn)
+    cache.check_status(sparq.DEV_CACHE_FULL)
+    assert cache.seq_lens.cpu().tolist() == [96, 96]
+    assert torch.equal(cache.K[0], K0[0]) and (cache.K[1, :, 95] == 1).all()
+
+
+def test_host_errors_launch_nothing():
+    q, K, V, seq = _small()
+    cache = H.DeviceCache(K, V, seq)
+    out = torch.empty(2, 4, 128, dtype=torch.float16, device="cuda")
+    for r, k, code in ((0, 4, sparq.ERR_BAD_RK), (129, 4, sparq.ERR_BAD_RK), (4, -1, sparq.ERR_BAD_RK),
+                       (4, sparq.K_MAX + 1, sparq.ERR_BAD_RK)):
+        with pytest.raises(sparq.SparqError) as e:
+            sparq.sparq_decode(q.cuda(), cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, r, k, out)
+        assert e.value.code == code
+    with pytest.raises(sparq.SparqError) as e:    # 3 query heads over 2 KV heads
+        sparq.sparq_decode(q[:, :3].contiguous().cuda(), cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens,
+                           4, 4, out[:, :3].contiguous())
+    assert e.value.code == sparq.ERR_BAD_SHAPE
+    assert sparq.sparq_max_seq_len() >= 32800
+
+
+# ------------------------------------------------------------------ host-buffer step
+def test_step_host_matches_device_step():
+    c = synth.make_case("c4", B=2, n_steps=2, ragged=(500, 900), Hq=8, Hkv=2, backend="numpy")
+    a = H.DeviceCache(c.K, c.V, c.seq_lens)
+    b = H.DeviceCache(c.K, c.V, c.seq_lens)
+    staging = torch.empty(sparq.sparq_step_host_staging_bytes(c.B, c.Hq, c.Hkv, c.d), dtype=torch.uint8, device="cuda")
+    out_host = torch.empty(c.B, c.Hq, c.d, dtype=torch.float16).pin_memory()
+    for i in range(c.n_steps):
+        a.append(c.k_steps[i], c.v_steps[i])
+        ref = a.decode(c.q_steps[i], c.r, c.k)
+        sparq.sparq_step_host(c.q_steps[i].pin_memory(), c.k_steps[i].pin_memory(), c.v_steps[i].pin_memory(),
+                              b.K, b.Kt, b.V, b.vsum, b.vbar, b.seq_lens, c.r, c.k, out_host, staging, b.status)
+        np.testing.assert_array_equal(out_host.numpy().astype(np.float64), ref["out"])
+    assert torch.equal(a.Kt, b.Kt) and torch.equal(a.seq_lens, b.seq_lens)
