@@ -170,10 +170,10 @@ def test_repeat_launches_are_bitwise_identical():
 
 
 def test_permuting_positions_permutes_the_selection():
-    q, K, V, seq = _small(B=1, Hq=2, Hkv=1, S=300)
+    q, K, V, seq = _small(B=1, Hq=2, Hkv=1, S=304, n=[300])
     cache = H.DeviceCache(K, V, seq)
     base = cache.decode(q, 16, 24)
-    perm = torch.randperm(300, generator=torch.Generator().manual_seed(3))
+    perm = torch.cat([torch.randperm(300, generator=torch.Generator().manual_seed(3)), torch.arange(300, 304)])
     cache2 = H.DeviceCache(K[:, :, perm], V[:, :, perm], seq)
     res = cache2.decode(q, 16, 24)
     for h in range(2):
