@@ -62,7 +62,9 @@ enum {
     SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds what the kernels' on-chip score buffer holds   */
     SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
     SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */
-    SPARQ_DEV_CACHE_FULL = 17    /* device: append with seq_lens[b] == S_max; nothing written    */
+    SPARQ_DEV_CACHE_FULL = 17,   /* device: append with seq_lens[b] == S_max; nothing written    */
+    SPARQ_DEV_TIMEOUT = 18       /* device: an asynchronous copy did not land within the bounded wait;
+                                    that out row is zero                                        */
 };
 
 /* Human-readable name of a status code (static string, never NULL). */

@@ -1,0 +1,131 @@
+// The C ABI of include/sparq.h: argument validation and kernel launches.  Nothing here
+// allocates device memory or synchronises, except sparq_step_host which waits for its stream.
+#include "kernels.h"
+
+namespace {
+
+using namespace sparq;
+
+int device_smem_optin() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
+    return v;
+}
+
+bool bad_common(int B, int Hq, int Hkv, int d, int S_max) {
+    return B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || d != SPARQ_HEAD_DIM || S_max < 8 || S_max % 8 != 0;
+}
+
+int rc(cudaError_t e) { return e == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* sparq_status_string(int code) {
+    switch (code) {
+        case SPARQ_OK: return "SPARQ_OK";
+        case SPARQ_ERR_NULL_POINTER: return "SPARQ_ERR_NULL_POINTER";
+        case SPARQ_ERR_BAD_SHAPE: return "SPARQ_ERR_BAD_SHAPE";
+        case SPARQ_ERR_BAD_RK: return "SPARQ_ERR_BAD_RK";
+        case SPARQ_ERR_WORKSPACE: return "SPARQ_ERR_WORKSPACE";
+        case SPARQ_ERR_TOO_LONG: return "SPARQ_ERR_TOO_LONG";
+        case SPARQ_ERR_CUDA: return "SPARQ_ERR_CUDA";
+        case SPARQ_DEV_BAD_SEQ_LEN: return "SPARQ_DEV_BAD_SEQ_LEN";
+        case SPARQ_DEV_CACHE_FULL: return "SPARQ_DEV_CACHE_FULL";
+        case SPARQ_DEV_TIMEOUT: return "SPARQ_DEV_TIMEOUT";
+        default: return "SPARQ_UNKNOWN_STATUS";
+    }
+}
+
+int sparq_max_seq_len(void) {
+    long avail = (long)device_smem_optin() - (long)decode_static_smem() - (long)decode_dynamic_smem(0) - 1024;
+    if (avail <= 0) return 0;
+    long s = (avail / 4) & ~7L;
+    long cap = decode_max_positions();
+    return (int)(s < cap ? s : cap);
+}
+
+int sparq_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                      sparq_half* Kt, float* vsum, sparq_half* vbar,
+                      int B, int Hkv, int d, int S_max, int32_t* status, void* stream) {
+    if (!K || !V || !seq_lens || !Kt || !vsum || !vbar) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hkv, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    return rc(launch_cache_build(K, V, seq_lens, Kt, vsum, vbar, B, Hkv, S_max, status, (cudaStream_t)stream));
+}
+
+int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
+                       sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
+                       int32_t* seq_lens, int B, int Hkv, int d, int S_max, int32_t* status, void* stream) {
+    if (!k_new || !v_new || !K || !Kt || !V || !vsum || !vbar || !seq_lens) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hkv, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    return rc(launch_cache_append(k_new, v_new, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, S_max, status,
+                                  (cudaStream_t)stream));
+}
+
+size_t sparq_workspace_bytes(int, int, int, int, int, int, int) { return 0; }
+
+int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                 const sparq_half* vbar, const int32_t* seq_lens,
+                 int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                 sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    (void)workspace; (void)workspace_bytes;
+    if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
+    if (S_max > sparq_max_seq_len()) return SPARQ_ERR_TOO_LONG;
+    return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
+                                  status, (cudaStream_t)stream));
+}
+
+size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {
+    if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
+    return dense_scratch_bytes(B, Hq, Hkv, S_max);
+}
+
+int dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                 int B, int Hq, int Hkv, int d, int S_max, sparq_half* out,
+                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (!q || !K || !V || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    const size_t need = dense_scratch_bytes(B, Hq, Hkv, S_max);
+    if (need && (!workspace || workspace_bytes < need)) return SPARQ_ERR_WORKSPACE;
+    return rc(launch_dense_decode(q, K, V, seq_lens, B, Hq, Hkv, S_max, out, (float*)workspace, status,
+                                  (cudaStream_t)stream));
+}
+
+size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d) {
+    if (B < 1 || Hq < 1 || Hkv < 1 || d < 1) return 0;
+    return ((size_t)2 * B * Hq * d + (size_t)2 * B * Hkv * d) * sizeof(sparq_half);
+}
+
+int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, const sparq_half* v_new_host,
+                    sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
+                    int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                    sparq_half* out_host, void* staging, size_t staging_bytes, int32_t* status, void* stream) {
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (!staging || staging_bytes < sparq_step_host_staging_bytes(B, Hq, Hkv, d)) return SPARQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t nq = (size_t)B * Hq * d, nkv = (size_t)B * Hkv * d;
+    sparq_half* q_dev = (sparq_half*)staging;
+    sparq_half* out_dev = q_dev + nq;
+    sparq_half* k_dev = out_dev + nq;
+    sparq_half* v_dev = k_dev + nkv;
+    if (cudaMemcpyAsync(q_dev, q_host, nq * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(k_dev, k_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(v_dev, v_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return SPARQ_ERR_CUDA;
+    int code = sparq_cache_append(k_dev, v_dev, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, d, S_max, status, stream);
+    if (code != SPARQ_OK) return code;
+    code = sparq_decode(q_dev, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, out_dev, nullptr, nullptr, nullptr,
+                        nullptr, 0, status, stream);
+    if (code != SPARQ_OK) return code;
+    if (cudaMemcpyAsync(out_host, out_dev, nq * sizeof(sparq_half), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SPARQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA;
+}
+
+}  // extern "C"

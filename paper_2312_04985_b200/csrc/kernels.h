@@ -1,0 +1,35 @@
+// Internal launch interfaces between the kernel files and the C ABI (api.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "sparq.h"
+
+namespace sparq {
+
+// sparq_decode.cu
+size_t decode_static_smem();
+size_t decode_dynamic_smem(int S_max);
+int decode_max_positions();
+cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                                const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
+                                int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                int32_t* status, cudaStream_t stream);
+
+// dense_decode.cu
+int dense_splits(int B, int Hkv, int S_max);
+size_t dense_scratch_bytes(int B, int Hq, int Hkv, int S_max);
+cudaError_t launch_dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                                int B, int Hq, int Hkv, int S_max, sparq_half* out, float* scratch, int32_t* status,
+                                cudaStream_t stream);
+
+// cache.cu
+cudaError_t launch_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens, sparq_half* Kt,
+                               float* vsum, sparq_half* vbar, int B, int Hkv, int S_max, int32_t* status,
+                               cudaStream_t stream);
+cudaError_t launch_cache_append(const sparq_half* k_new, const sparq_half* v_new, sparq_half* K, sparq_half* Kt,
+                                sparq_half* V, float* vsum, sparq_half* vbar, int32_t* seq_lens, int B, int Hkv,
+                                int S_max, int32_t* status, cudaStream_t stream);
+
+}  // namespace sparq
