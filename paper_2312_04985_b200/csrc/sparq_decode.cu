@@ -31,11 +31,31 @@ constexpr int STAGE_BYTES = RB * CH * 2;
 constexpr int RING_BYTES = STAGES * STAGE_BYTES;
 constexpr int HIST_BINS = 2048;
 constexpr int BM_WORDS = 2048;           // bitmap capacity: 65536 positions
-constexpr int RG = 4;                    // gathered rows in flight per half-warp
+constexpr int RG = 8;                    // gathered rows in flight per half-warp
+constexpr int CAND_MAX = 256;            // threshold-band positions the quick fp64 re-decision handles
 constexpr int WAIT_LIMIT = 1 << 22;      // polls before a copy is declared lost
 
-static_assert(HIST_BINS * 4 + 2 * BM_WORDS * 4 + NHW * (D + 2) * 4 <= RING_BYTES, "a4/a5 scratch must fit the ring");
+static_assert(HIST_BINS * 4 + 2 * BM_WORDS * 4 + NHW * (D + 2) * 4 + CAND_MAX * 12 <= RING_BYTES, "a4/a5 scratch must fit the ring");
+static_assert(CAND_MAX <= NT, "one thread per band candidate");
 static_assert(NT >= D && HIST_BINS % NT == 0, "thread mapping");
+
+// Optional per-phase cycle counters (thread 0 of every CTA, summed over CTAs); compiled in only
+// with -DSPARQ_PHASE_CLOCKS for tuning, never in the shipped library.
+#ifdef SPARQ_PHASE_CLOCKS
+__device__ unsigned long long g_phase_clocks[16];
+#define PHASE_INIT() long long t_prev_ = clock64()
+#define PHASE_MARK(i)                                                                     \
+    do {                                                                                  \
+        if (threadIdx.x == 0) {                                                           \
+            long long t_now_ = clock64();                                                 \
+            atomicAdd(&g_phase_clocks[i], (unsigned long long)(t_now_ - t_prev_));        \
+            t_prev_ = t_now_;                                                             \
+        }                                                                                 \
+    } while (0)
+#else
+#define PHASE_INIT()
+#define PHASE_MARK(i)
+#endif
 
 struct DecodeShared {
     double qd[D];                 // tie path only: selected query components * 2^1008, in i1 order
@@ -45,9 +65,10 @@ struct DecodeShared {
     uint16_t qh[D + RB];          // selected query components (fp16 bits) in i1 order
     int32_t i2[SPARQ_K_MAX];
     uint64_t full[STAGES];        // mbarriers: stage s has landed
-    float red[NW];
-    uint32_t redu[NW];
+    float red[2 * NW];
+    uint32_t redu[2 * NW];
     uint32_t res[4];
+    uint32_t band[4];             // [0] keys in [lo, edge), [1] keys in [edge, hi], [2] candidate list length
     float inv_tau, l1_sel;
 };
 
@@ -70,6 +91,17 @@ __device__ __forceinline__ uint32_t block_max_u32(uint32_t v, uint32_t* red) {
 #pragma unroll
     for (int w = 0; w < NW; ++w) t = max(t, red[w]);
     return t;
+}
+// Two block-wide maxima with one pair of barriers.  red: 2*NW words.
+__device__ __forceinline__ void block_max2_u32(uint32_t& a, uint32_t& b, uint32_t* red) {
+    a = __reduce_max_sync(FULL, a);
+    b = __reduce_max_sync(FULL, b);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = a; red[NW + (threadIdx.x >> 5)] = b; }
+    __syncthreads();
+    a = 0; b = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { a = max(a, red[w]); b = max(b, red[NW + w]); }
 }
 __device__ __forceinline__ uint32_t block_sum_u32(uint32_t v, uint32_t* red) {
     v = __reduce_add_sync(FULL, v);
@@ -126,6 +158,12 @@ __device__ __forceinline__ void zero_hist(uint32_t* hist) {
     for (int i = threadIdx.x; i < HIST_BINS / 4; i += NT) h4[i] = make_uint4(0, 0, 0, 0);
 }
 
+__device__ __forceinline__ float ex2(float x) {            // 2^x, 2 ulp; exact enough for softmax weights
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // d = a * b + d with fp16 a, b and fp32 d: the product is exact, one rounding (sm_100 mixed FMA).
 __device__ __forceinline__ void fma_h(float& d, uint16_t a, uint16_t b) {
     asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(d) : "h"(a), "h"(b));
@@ -151,7 +189,7 @@ __device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const Deco
     return acc;
 }
 
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NT, 3)
 sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                     const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
                     const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
@@ -166,6 +204,8 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     uint32_t* bm_sel = hist + HIST_BINS;                                  // bit t: position t is selected
     uint32_t* bm_tie = bm_sel + BM_WORDS;                                 // bit t: exact fp64 tie at the threshold
     float* merge = reinterpret_cast<float*>(bm_tie + BM_WORDS);
+    unsigned long long* cand_val = reinterpret_cast<unsigned long long*>(merge + NHW * (D + 2));   // band candidates' fp64 keys
+    int32_t* cand_pos = reinterpret_cast<int32_t*>(cand_val + CAND_MAX);                           // and positions
     __shared__ DecodeShared sh;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -182,6 +222,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         return;
     }
     const int k_eff = min(k, n);
+    PHASE_INIT();
     if (tid == 0) {
 #pragma unroll
         for (int s = 0; s < STAGES; ++s) mbar_init(&sh.full[s], 1);
@@ -232,6 +273,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     const float inv_tau = sh.inv_tau;
 
     float alpha = 0.f;
+    PHASE_MARK(0);
     if (k_eff > 0) {
         // -------------------------------------------------------------- a2: stream r rows of Kt
         const sparq_half* Kt_head = Kt + kv_head * (size_t)D * S_max;
@@ -239,16 +281,19 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         const int n_chunks = (n8 + CH - 1) / CH;
         const int nb = r_pad / RB;
         const int total = n_chunks * nb;
-        auto issue = [&](int it, int s) {                    // thread 0: fill slot s with iteration `it`
+        // Warp 0 refills a slot: lane 0 arms the barrier, then lanes 0..rows-1 each issue one row's
+        // copy (one thread can only start a bulk copy every few hundred cycles; lanes overlap).
+        auto issue = [&](int it, int s) {
             const int c = it / nb, jb = (it - c * nb) * RB;
             const uint32_t bytes = (uint32_t)min(CH, n8 - c * CH) * 2u;
             const int rows = min(RB, r - jb);
-            mbar_expect_tx(&sh.full[s], bytes * rows);
-            for (int u = 0; u < rows; ++u)
-                bulk_g2s(ring + s * STAGE_BYTES + u * (CH * 2), Kt_head + (size_t)sh.i1[jb + u] * S_max + c * CH, bytes,
+            if (lane == 0) mbar_expect_tx(&sh.full[s], bytes * rows);
+            __syncwarp();
+            if (lane < rows)
+                bulk_g2s(ring + s * STAGE_BYTES + lane * (CH * 2), Kt_head + (size_t)sh.i1[jb + lane] * S_max + c * CH, bytes,
                          &sh.full[s]);
         };
-        if (tid == 0) for (int it = 0; it < min(STAGES, total); ++it) issue(it, it);
+        if (warp == 0) for (int it = 0; it < min(STAGES, total); ++it) issue(it, it);
 
         uint32_t kmax = 0;
         __half2 mx = __float2half2_rn(0.f);                  // largest |K| among the valid streamed values
@@ -283,7 +328,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                 }
                 ok = __syncthreads_and(ok);                  // slot s fully consumed (or a wait gave up)
                 if (!ok) break;
-                if (tid == 0 && it + STAGES < total) issue(it + STAGES, s);
+                if (warp == 0 && it + STAGES < total) issue(it + STAGES, s);
                 if (++s == STAGES) { s = 0; parity ^= 1u; }
             }
             if (!ok) break;
@@ -306,9 +351,11 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
             if (idx_k) for (int j = tid; j < k; j += NT) idx_k[(size_t)bh * k + j] = -1;
             return;
         }
-        kmax = block_max_u32(kmax, sh.redu);                 // barriers: keys complete, ring is dead
+        PHASE_MARK(1);
+        uint32_t kabs_bits = __float_as_uint(fmaxf(__low2float(mx), __high2float(mx)));
+        block_max2_u32(kmax, kabs_bits, sh.redu);            // barriers: keys complete, ring is dead
         const float vmax = unkey32(kmax);
-        const float kabs = __uint_as_float(block_max_u32(__float_as_uint(fmaxf(__low2float(mx), __high2float(mx))), sh.redu));
+        const float kabs = __uint_as_float(kabs_bits);
         // |fp32 chain - exact sum| <= ((1+u)^r - 1) sum_j |q_j K_tj| <= 1.02 r u ||q[i1]||_1 max|K|,  u = 2^-24
         const float twoB = 2.f * (1.02f * (float)r * 5.9604645e-8f * sh.l1_sel * kabs) + 1e-37f * (float)(kabs > 0.f);
 
@@ -338,73 +385,99 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                 if (ceq == need) break;                      // the whole bin is selected: no need to split it
             }
         }
+        PHASE_MARK(2);
         const uint32_t edge = prefix;                        // unprocessed low bits are zero
         const uint32_t over = ceq - need;
         const float edge_val = unkey32(edge);
         const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
 
         // -------------------------------------------------------------- a3 + bitmap of the selection
-        // Softmax denominator, the speculative selection key >= edge as a bitmap, and how many keys
-        // lie within 2B below / above the edge.
+        // Softmax denominator, the speculative selection key >= edge as a bitmap, and the positions
+        // whose key lies within 2B of the edge (counted on each side, listed while the list has room).
         const int nwords = (n + 31) >> 5;
         const float c1 = inv_tau * LOG2E;
+        if (tid < 4) sh.band[tid] = 0;
+        __syncthreads();
         float zpart = 0.f;
-        uint32_t cnt_lo = 0, cnt_hi = 0;
         for (int wi = warp; wi < nwords; wi += NW) {
             const int t = (wi << 5) + lane;
             const bool valid = t < n;
             const uint32_t u = valid ? keys[t] : 0u;
-            zpart += valid ? exp2f((unkey32(u) - vmax) * c1) : 0.f;
+            zpart += valid ? ex2((unkey32(u) - vmax) * c1) : 0.f;
             const bool ge = valid && u >= edge;
             const unsigned g = __ballot_sync(FULL, ge);
             if (lane == 0) bm_sel[wi] = g;
-            cnt_hi += (ge && u <= hi_key);
-            cnt_lo += (valid && !ge && u >= lo_key);
+            if (valid && u >= lo_key && u <= hi_key) {       // rare
+                atomicAdd(&sh.band[ge ? 1 : 0], 1u);
+                const uint32_t slot = atomicAdd(&sh.band[2], 1u);
+                if (slot < CAND_MAX) cand_pos[slot] = t;
+            }
         }
-        const float Z = block_sum(zpart, sh.red);
-        cnt_lo = block_sum_u32(cnt_lo, sh.redu);
-        cnt_hi = block_sum_u32(cnt_hi, sh.redu);             // barriers also publish the bitmap
+        const float Z = block_sum(zpart, sh.red);            // barriers also publish the bitmap and the band
+        const uint32_t cnt_lo = sh.band[0], cnt_hi = sh.band[1], n_cand = sh.band[2];
+        PHASE_MARK(3);
         uint32_t need_tie = 0;
         if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
-            // Rare: fp32 sums on both sides of the threshold are closer to it than their error bound
-            // (or tie).  The cnt_lo + cnt_hi positions in the band compete for cnt_hi - over places by
-            // their fp64 sums: radix select over their 64-bit keys, 8 passes of 8 bits, then rebuild
-            // the bitmap.  Equal fp64 sums at the threshold go to the lowest positions.
-            unsigned long long p64 = 0, m64 = 0;
-            uint32_t need64 = cnt_hi - over;
-#pragma unroll 1
-            for (int shift = 56; shift >= 0; shift -= 8) {
-                zero_hist(hist);
+            // fp32 sums on both sides of the threshold are closer to it than their error bound (or
+            // tie).  The n_cand positions in the band compete for cnt_hi - over places by their fp64
+            // sums of exact products; equal fp64 sums go to the lowest positions.
+            const uint32_t need64 = cnt_hi - over;
+            if (n_cand <= CAND_MAX) {
+                // few candidates: one thread each, rank by counting, then patch their bitmap bits
+                unsigned long long v = 0;
+                int t = 0;
+                if (tid < n_cand) { t = cand_pos[tid]; v = key64(dot64_at(Kt_head, sh, S_max, r, t)); cand_val[tid] = v; }
                 __syncthreads();
-                for (int t = tid; t < n; t += NT) {
-                    const uint32_t u = keys[t];
-                    if (u >= lo_key && u <= hi_key) {
-                        const unsigned long long v = key64(dot64_at(Kt_head, sh, S_max, r, t));
-                        if ((v & m64) == p64) atomicAdd(&hist[(uint32_t)(v >> shift) & 255u], 1u);
+                if (tid < n_cand) {
+                    uint32_t rank = 0;
+                    for (uint32_t i = 0; i < n_cand; ++i) {
+                        const unsigned long long vi = cand_val[i];
+                        rank += (vi > v) || (vi == v && cand_pos[i] < t);
                     }
+                    if (rank < need64) atomicOr(&bm_sel[t >> 5], 1u << (t & 31));
+                    else atomicAnd(&bm_sel[t >> 5], ~(1u << (t & 31)));
                 }
                 __syncthreads();
-                find_bin(hist, need64, sh.redu, sh.res);
-                p64 |= (unsigned long long)sh.res[0] << shift;
-                m64 |= 255ull << shift;
-                need64 -= sh.res[1];
-            }
-            need_tie = need64;
-            for (int wi = warp; wi < nwords; wi += NW) {
-                const int t = (wi << 5) + lane;
-                const uint32_t u = t < n ? keys[t] : 0u;
-                bool s_ = t < n && u > hi_key, tie = false;
-                if (t < n && u >= lo_key && u <= hi_key) {
-                    const unsigned long long v = key64(dot64_at(Kt_head, sh, S_max, r, t));
-                    s_ = v > p64;
-                    tie = v == p64;
+            } else {
+                // many candidates (degenerate inputs, e.g. constant keys): radix select over their
+                // 64-bit keys, 8 passes of 8 bits, then rebuild the bitmap
+                unsigned long long p64 = 0, m64 = 0;
+                uint32_t left = need64;
+#pragma unroll 1
+                for (int shift = 56; shift >= 0; shift -= 8) {
+                    zero_hist(hist);
+                    __syncthreads();
+                    for (int t = tid; t < n; t += NT) {
+                        const uint32_t u = keys[t];
+                        if (u >= lo_key && u <= hi_key) {
+                            const unsigned long long v = key64(dot64_at(Kt_head, sh, S_max, r, t));
+                            if ((v & m64) == p64) atomicAdd(&hist[(uint32_t)(v >> shift) & 255u], 1u);
+                        }
+                    }
+                    __syncthreads();
+                    find_bin(hist, left, sh.redu, sh.res);
+                    p64 |= (unsigned long long)sh.res[0] << shift;
+                    m64 |= 255ull << shift;
+                    left -= sh.res[1];
                 }
-                const unsigned g = __ballot_sync(FULL, s_), te = __ballot_sync(FULL, tie);
-                if (lane == 0) { bm_sel[wi] = g; bm_tie[wi] = te; }
+                need_tie = left;
+                for (int wi = warp; wi < nwords; wi += NW) {
+                    const int t = (wi << 5) + lane;
+                    const uint32_t u = t < n ? keys[t] : 0u;
+                    bool s_ = t < n && u > hi_key, tie = false;
+                    if (t < n && u >= lo_key && u <= hi_key) {
+                        const unsigned long long v = key64(dot64_at(Kt_head, sh, S_max, r, t));
+                        s_ = v > p64;
+                        tie = v == p64;
+                    }
+                    const unsigned g = __ballot_sync(FULL, s_), te = __ballot_sync(FULL, tie);
+                    if (lane == 0) { bm_sel[wi] = g; bm_tie[wi] = te; }
+                }
+                __syncthreads();
             }
-            __syncthreads();
         }
 
+        PHASE_MARK(4);
         // ascending list of selected positions from the bitmap(s)
         uint32_t carry_tie = 0, carry_sel = 0;
         for (int base = 0; base < nwords; base += NT) {
@@ -433,9 +506,10 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         __syncthreads();
         // alpha = approximate-score mass of the selected set (Step 3)
         float apart = 0.f;
-        for (int j = tid; j < k_eff; j += NT) apart += exp2f((unkey32(keys[sh.i2[j]]) - vmax) * c1);
+        for (int j = tid; j < k_eff; j += NT) apart += ex2((unkey32(keys[sh.i2[j]]) - vmax) * c1);
         alpha = block_sum(apart, sh.red) / Z;
 
+        PHASE_MARK(5);
         // -------------------------------------------------------------- a5: gather k rows of K and V
         const int hw = tid >> 4, l16 = tid & 15;
         const float qscale = rsqrtf((float)D) * LOG2E;
@@ -473,13 +547,13 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
             }
             const float mn = fmaxf(m, bmax);
             if (mn > -CUDART_INF_F) {
-                const float sc = exp2f(m - mn);
+                const float sc = ex2(m - mn);
                 l *= sc;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] *= sc;
 #pragma unroll
                 for (int u = 0; u < RG; ++u) {
-                    const float p = exp2f(z[u] - mn);
+                    const float p = ex2(z[u] - mn);
                     l += p;
                     const __half2* vh = reinterpret_cast<const __half2*>(&vv[u]);
 #pragma unroll
@@ -492,6 +566,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                 m = mn;
             }
         }
+        PHASE_MARK(6);
         // merge the half-warps' partial softmax states
         float* mg = merge + hw * (D + 2);
 #pragma unroll
@@ -511,7 +586,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
             float L = 0.f, s = 0.f;
 #pragma unroll
             for (int w = 0; w < NHW; ++w) {
-                const float sc = exp2f(merge[w * (D + 2) + D] - M);
+                const float sc = ex2(merge[w * (D + 2) + D] - M);
                 L = fmaf(merge[w * (D + 2) + D + 1], sc, L);
                 s = fmaf(merge[w * (D + 2) + tid], sc, s);
             }
@@ -521,9 +596,19 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     }
     if (tid == 0 && alpha_out) alpha_out[bh] = alpha;
     if (idx_k) for (int j = tid; j < k; j += NT) idx_k[(size_t)bh * k + j] = (j < k_eff) ? sh.i2[j] : -1;
+    PHASE_MARK(7);
 }
 
 }  // namespace
+
+#ifdef SPARQ_PHASE_CLOCKS
+extern "C" int sparq_debug_phase_clocks(unsigned long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    if (out16 && cudaMemcpyFromSymbol(out16, g_phase_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_phase_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+#endif
 
 size_t decode_static_smem() { return sizeof(DecodeShared); }
 size_t decode_dynamic_smem(int S_max) { return (size_t)RING_BYTES + (size_t)S_max * sizeof(uint32_t); }
