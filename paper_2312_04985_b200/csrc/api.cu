@@ -1,5 +1,8 @@
 // The C ABI of include/sparq.h: argument validation and kernel launches.  Nothing here
 // allocates device memory or synchronises, except sparq_step_host which waits for its stream.
+#include <stdlib.h>
+#include <string.h>
+
 #include "kernels.h"
 
 namespace {
@@ -15,6 +18,23 @@ int device_smem_optin() {
 
 bool bad_common(int B, int Hq, int Hkv, int d, int S_max) {
     return B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || d != SPARQ_HEAD_DIM || S_max < 8 || S_max % 8 != 0;
+}
+
+int device_sm_count() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return v;
+}
+
+// SPARQ_DECODE_PLAN=simple|pipe forces one of the two sparq_decode kernels (tests and tuning);
+// unset or anything else: the persistent pipelined kernel whenever its buffers fit.
+int forced_plan() {
+    const char* e = getenv("SPARQ_DECODE_PLAN");
+    if (!e) return 0;
+    if (!strcmp(e, "simple")) return 1;
+    if (!strcmp(e, "pipe")) return 2;
+    return 0;
 }
 
 int rc(cudaError_t e) { return e == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA; }
@@ -76,6 +96,12 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
     if (S_max > sparq_max_seq_len()) return SPARQ_ERR_TOO_LONG;
+    const int plan = forced_plan();
+    const bool fits = pipe_fits(S_max, device_smem_optin());
+    if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
+    if (fits && plan != 1)
+        return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
+                                           alpha, status, device_sm_count(), (cudaStream_t)stream));
     return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
                                   status, (cudaStream_t)stream));
 }

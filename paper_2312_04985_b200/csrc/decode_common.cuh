@@ -1,0 +1,432 @@
+// Building blocks shared by the two sparq_decode kernels (the one-CTA-per-head kernel and the
+// persistent warp-specialised one): thread-group reductions, the streamed fp32 score chain, and
+// the whole "post" phase -- top-k select with exact re-decision of the threshold band, softmax
+// statistics, ascending index list, K/V row gather with online softmax, and the v_bar combine.
+#pragma once
+#include "common.cuh"
+
+namespace sparq {
+
+constexpr int HIST_BINS = 2048;
+constexpr int CAND_MAX = 256;            // threshold-band positions the quick fp64 re-decision handles
+constexpr int RG = 8;                    // gathered rows in flight per half-warp
+constexpr int WAIT_LIMIT = 1 << 22;      // polls before an asynchronous copy is declared lost
+
+// A group of NT_ consecutive threads (whole warps) that synchronises on its own barrier.
+// BAR_ == 0: the whole CTA (__syncthreads); otherwise named barrier BAR_.
+template <int NT_, int BAR_>
+struct Group {
+    static constexpr int NT = NT_, NW = NT_ / 32, NHW = NT_ / 16;
+    static __device__ __forceinline__ void sync() {
+        if constexpr (BAR_ == 0) __syncthreads();
+        else asm volatile("bar.sync %0, %1;" ::"n"(BAR_), "n"(NT_) : "memory");
+    }
+};
+
+// What the later stages need to know about one (batch, query head) unit; filled by stage a1.
+struct HeadMeta {
+    float qf[D];                  // q as fp32
+    int32_t i1[D];                // selected components, ascending
+    uint32_t rkey[D];             // a1 scratch: ranking keys
+    uint16_t qh[D + 8];           // selected components' fp16 bits in i1 order, zero padded
+    int32_t bh, n, k_eff, valid;
+    float inv_tau, l1_sel;
+};
+
+// Shared-memory scratch of one post phase.
+struct PostScratch {
+    uint32_t* hist;               // [HIST_BINS]
+    uint32_t* bm_sel;             // [ceil(n/32)] bit t: position t is selected
+    uint32_t* bm_tie;             // [ceil(n/32)] bit t: exact fp64 tie at the threshold (degenerate path)
+    float* merge;                 // [NHW * (D + 2)]
+    unsigned long long* cand_val; // [CAND_MAX]
+    int32_t* cand_pos;            // [CAND_MAX]
+    int32_t* i2;                  // [SPARQ_K_MAX]
+    float* red;                   // [2 * NW]
+    uint32_t* redu;               // [2 * NW]
+    uint32_t* res;                // [4]
+    uint32_t* band;               // [4]
+};
+// bytes of the scratch that may alias a dead buffer (everything except i2 and the small arrays)
+__host__ __device__ constexpr size_t post_scratch_bytes(int nhw, int bm_words) {
+    return (size_t)HIST_BINS * 4 + 2 * (size_t)bm_words * 4 + (size_t)nhw * (D + 2) * 4 + (size_t)CAND_MAX * 12;
+}
+__device__ __forceinline__ void carve_post_scratch(PostScratch& sc, unsigned char* base, int nhw, int bm_words) {
+    sc.hist = reinterpret_cast<uint32_t*>(base);
+    sc.bm_sel = sc.hist + HIST_BINS;
+    sc.bm_tie = sc.bm_sel + bm_words;
+    sc.merge = reinterpret_cast<float*>(sc.bm_tie + bm_words);
+    sc.cand_val = reinterpret_cast<unsigned long long*>(sc.merge + nhw * (D + 2));
+    sc.cand_pos = reinterpret_cast<int32_t*>(sc.cand_val + CAND_MAX);
+}
+
+__device__ __forceinline__ float ex2(float x) {            // 2^x, 2 ulp; exact enough for softmax weights
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// d = a * b + d with fp16 a, b and fp32 d: the product is exact, one rounding (sm_100 mixed FMA).
+__device__ __forceinline__ void fma_h(float& d, uint16_t a, uint16_t b) {
+    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(d) : "h"(a), "h"(b));
+}
+
+// One Kt row vector (8 positions) times one query component into the 8 running sums; mx tracks
+// the largest |K| seen (four independent chains).
+__device__ __forceinline__ void row_fma(float (&acc)[8], __half2 (&mx)[4], uint4 v, uint16_t qj) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        fma_h(acc[2 * e], (uint16_t)(w[e] & 0xffffu), qj);
+        fma_h(acc[2 * e + 1], (uint16_t)(w[e] >> 16), qj);
+        mx[e] = __hmax2(mx[e], __habs2(*reinterpret_cast<const __half2*>(&w[e])));
+    }
+}
+__device__ __forceinline__ float mx_to_float(const __half2 (&mx)[4]) {
+    const __half2 a = __hmax2(__hmax2(mx[0], mx[1]), __hmax2(mx[2], mx[3]));
+    return fmaxf(__low2float(a), __high2float(a));
+}
+
+// ---- group-wide reductions in a fixed order (bitwise reproducible run to run) -------------
+template <class G>
+__device__ __forceinline__ float group_sum(float v, float* red, int gtid) {
+    v = warp_sum(v);
+    G::sync();
+    if ((gtid & 31) == 0) red[gtid >> 5] = v;
+    G::sync();
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < G::NW; ++w) t += red[w];
+    return t;
+}
+template <class G>
+__device__ __forceinline__ void group_sum2(float& a, float& b, float* red, int gtid) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    G::sync();
+    if ((gtid & 31) == 0) { red[gtid >> 5] = a; red[G::NW + (gtid >> 5)] = b; }
+    G::sync();
+    a = 0.f; b = 0.f;
+#pragma unroll
+    for (int w = 0; w < G::NW; ++w) { a += red[w]; b += red[G::NW + w]; }
+}
+template <class G>
+__device__ __forceinline__ void group_max2_u32(uint32_t& a, uint32_t& b, uint32_t* red, int gtid) {
+    a = __reduce_max_sync(FULL, a);
+    b = __reduce_max_sync(FULL, b);
+    G::sync();
+    if ((gtid & 31) == 0) { red[gtid >> 5] = a; red[G::NW + (gtid >> 5)] = b; }
+    G::sync();
+    a = 0; b = 0;
+#pragma unroll
+    for (int w = 0; w < G::NW; ++w) { a = max(a, red[w]); b = max(b, red[G::NW + w]); }
+}
+// Inclusive prefix sum over the group in thread order; *total receives the group-wide sum.
+template <class G>
+__device__ __forceinline__ uint32_t group_scan_incl(uint32_t v, uint32_t* red, uint32_t* total, int gtid) {
+    const int lane = gtid & 31, warp = gtid >> 5;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t x = __shfl_up_sync(FULL, v, o);
+        if (lane >= o) v += x;
+    }
+    G::sync();
+    if (lane == 31) red[warp] = v;
+    G::sync();
+    uint32_t before = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < G::NW; ++w) { if (w < warp) before += red[w]; tot += red[w]; }
+    *total = tot;
+    return v + before;
+}
+
+// One radix-select pass over an already filled histogram: find, from the top, the bin holding the
+// need-th largest candidate.  res[0] = bin, res[1] = candidates above it, res[2] = candidates in
+// it.  All threads of the group call; the result is valid after the trailing barrier.
+template <class G>
+__device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, uint32_t* red, uint32_t* res, int gtid) {
+    constexpr int PER = HIST_BINS / G::NT;
+    static_assert(HIST_BINS % G::NT == 0, "bins per thread");
+    const int top = HIST_BINS - 1 - gtid * PER;              // this thread's bins: top, top-1, ...
+    uint32_t c[PER], s = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { c[i] = hist[top - i]; s += c[i]; }
+    uint32_t total;
+    uint32_t incl = group_scan_incl<G>(s, red, &total, gtid);
+    uint32_t run = incl - s;
+    if (run < need && need <= incl) {
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            if (run + c[i] >= need) { res[0] = top - i; res[1] = run; res[2] = c[i]; break; }
+            run += c[i];
+        }
+    }
+    G::sync();
+}
+template <class G>
+__device__ __forceinline__ void zero_hist(uint32_t* hist, int gtid) {
+    uint4* h4 = reinterpret_cast<uint4*>(hist);
+    for (int i = gtid; i < HIST_BINS / 4; i += G::NT) h4[i] = make_uint4(0, 0, 0, 0);
+}
+
+// fp64 sum of the exact products of the selected query components with position t of the r
+// selected Kt rows, in i1 order: bit for bit the float64 oracle's accumulation.
+__device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t) {
+    double acc = 0.0;
+    for (int j = 0; j < r; ++j) {
+        const int c = hm.i1[j];
+        acc = fma(ldexp((double)hm.qf[c], 1008), h2d_scalar(Kt_head[(size_t)c * S_max + t]), acc);
+    }
+    return acc;
+}
+
+// Stages a4, a3, a5, a6 for one head, run by the thread group G (gtid = thread index in the group).
+//   keys[0..n): order-preserving keys of the fp32 approximate-score sums; kmax their maximum;
+//   kabs: largest |K| among the streamed values (error bound of the sums).
+// Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
+// group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
+template <class G>
+__device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, float kabs,
+                                           const PostScratch& sc, int r, int k, int S_max,
+                                           const sparq_half* __restrict__ Kt_head, const sparq_half* __restrict__ K_head,
+                                           const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
+                                           sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
+                                           float* __restrict__ alpha_out) {
+    const int lane = gtid & 31, warp = gtid >> 5;
+    const int n = hm.n, k_eff = hm.k_eff;
+    const float inv_tau = hm.inv_tau;
+    const float vmax = unkey32(kmax);
+    // |fp32 chain - exact sum| <= ((1+u)^r - 1) sum_j |q_j K_tj| <= 1.02 r u ||q[i1]||_1 max|K|,  u = 2^-24
+    const float twoB = 2.f * (1.02f * (float)r * 5.9604645e-8f * hm.l1_sel * kabs);
+
+    // -------------------------------------------------------------- a4: top-k select
+    // MSB radix select, 11 + 11 + 10 bits, leaving the loop as soon as a whole bin is wanted.
+    // Afterwards the k_eff largest keys are those >= edge, except that `over` too many keys equal
+    // edge when the fp32 sums tie at the threshold.
+    uint32_t prefix = 0, mask = 0, need = (uint32_t)k_eff, ceq = 0;
+    {
+        int shift = 32;
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            const int bits = pass < 2 ? 11 : 10;
+            shift -= bits;
+            zero_hist<G>(sc.hist, gtid);
+            G::sync();
+            for (int t = gtid; t < n; t += G::NT) {
+                const uint32_t u = keys[t];
+                if ((u & mask) == prefix) atomicAdd(&sc.hist[(u >> shift) & ((1u << bits) - 1)], 1u);
+            }
+            G::sync();
+            find_bin<G>(sc.hist, need, sc.redu, sc.res, gtid);
+            prefix |= sc.res[0] << shift;
+            mask |= ((1u << bits) - 1) << shift;
+            need -= sc.res[1];
+            ceq = sc.res[2];
+            if (ceq == need) break;                          // the whole bin is selected: no need to split it
+        }
+    }
+    const uint32_t edge = prefix;                            // unprocessed low bits are zero
+    const uint32_t over = ceq - need;
+    const float edge_val = unkey32(edge);
+    const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
+
+    // -------------------------------------------------------------- a3 + bitmap of the selection
+    // Softmax denominator, the speculative selection key >= edge as a bitmap, and the positions
+    // whose key lies within 2B of the edge (counted on each side, listed while the list has room).
+    const int nwords = (n + 31) >> 5;
+    const float c1 = inv_tau * LOG2E;
+    if (gtid < 4) sc.band[gtid] = 0;
+    G::sync();
+    float zpart = 0.f;
+    for (int wi = warp; wi < nwords; wi += G::NW) {
+        const int t = (wi << 5) + lane;
+        const bool valid = t < n;
+        const uint32_t u = valid ? keys[t] : 0u;
+        zpart += valid ? ex2((unkey32(u) - vmax) * c1) : 0.f;
+        const bool ge = valid && u >= edge;
+        const unsigned g = __ballot_sync(FULL, ge);
+        if (lane == 0) sc.bm_sel[wi] = g;
+        if (valid && u >= lo_key && u <= hi_key) {           // rare
+            atomicAdd(&sc.band[ge ? 1 : 0], 1u);
+            const uint32_t slot = atomicAdd(&sc.band[2], 1u);
+            if (slot < CAND_MAX) sc.cand_pos[slot] = t;
+        }
+    }
+    const float Z = group_sum<G>(zpart, sc.red, gtid);       // barriers also publish the bitmap and the band
+    const uint32_t cnt_lo = sc.band[0], cnt_hi = sc.band[1], n_cand = sc.band[2];
+    uint32_t need_tie = 0;
+    if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
+        // fp32 sums on both sides of the threshold are closer to it than their error bound (or
+        // tie).  The n_cand positions in the band compete for cnt_hi - over places by their fp64
+        // sums of exact products; equal fp64 sums go to the lowest positions.
+        const uint32_t need64 = cnt_hi - over;
+        if (n_cand <= CAND_MAX) {
+            // few candidates: one thread each, rank by counting, then patch their bitmap bits
+            static_assert(CAND_MAX <= G::NT, "one thread per band candidate");
+            unsigned long long v = 0;
+            int t = 0;
+            if (gtid < n_cand) { t = sc.cand_pos[gtid]; v = key64(dot64_at(Kt_head, hm, S_max, r, t)); sc.cand_val[gtid] = v; }
+            G::sync();
+            if (gtid < n_cand) {
+                uint32_t rank = 0;
+                for (uint32_t i = 0; i < n_cand; ++i) {
+                    const unsigned long long vi = sc.cand_val[i];
+                    rank += (vi > v) || (vi == v && sc.cand_pos[i] < t);
+                }
+                if (rank < need64) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
+                else atomicAnd(&sc.bm_sel[t >> 5], ~(1u << (t & 31)));
+            }
+            G::sync();
+        } else {
+            // many candidates (degenerate inputs, e.g. constant keys): radix select over their
+            // 64-bit keys, 8 passes of 8 bits, then rebuild the bitmap
+            unsigned long long p64 = 0, m64 = 0;
+            uint32_t left = need64;
+#pragma unroll 1
+            for (int shift = 56; shift >= 0; shift -= 8) {
+                zero_hist<G>(sc.hist, gtid);
+                G::sync();
+                for (int t = gtid; t < n; t += G::NT) {
+                    const uint32_t u = keys[t];
+                    if (u >= lo_key && u <= hi_key) {
+                        const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t));
+                        if ((v & m64) == p64) atomicAdd(&sc.hist[(uint32_t)(v >> shift) & 255u], 1u);
+                    }
+                }
+                G::sync();
+                find_bin<G>(sc.hist, left, sc.redu, sc.res, gtid);
+                p64 |= (unsigned long long)sc.res[0] << shift;
+                m64 |= 255ull << shift;
+                left -= sc.res[1];
+            }
+            need_tie = left;
+            for (int wi = warp; wi < nwords; wi += G::NW) {
+                const int t = (wi << 5) + lane;
+                const uint32_t u = t < n ? keys[t] : 0u;
+                bool s_ = t < n && u > hi_key, tie = false;
+                if (t < n && u >= lo_key && u <= hi_key) {
+                    const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t));
+                    s_ = v > p64;
+                    tie = v == p64;
+                }
+                const unsigned g = __ballot_sync(FULL, s_), te = __ballot_sync(FULL, tie);
+                if (lane == 0) { sc.bm_sel[wi] = g; sc.bm_tie[wi] = te; }
+            }
+            G::sync();
+        }
+    }
+
+    // ascending list of selected positions from the bitmap(s)
+    uint32_t carry_tie = 0, carry_sel = 0;
+    for (int base = 0; base < nwords; base += G::NT) {
+        const int wi = base + gtid;
+        uint32_t g = wi < nwords ? sc.bm_sel[wi] : 0u;
+        if (need_tie) {                                      // add the first need_tie tied positions
+            uint32_t e = wi < nwords ? sc.bm_tie[wi] : 0u, tot;
+            const uint32_t ce = __popc(e);
+            const uint32_t before = carry_tie + group_scan_incl<G>(ce, sc.redu, &tot, gtid) - ce;
+            const uint32_t allowed = before >= need_tie ? 0u : min(ce, need_tie - before);
+            while ((uint32_t)__popc(e) > allowed) e &= ~(0x80000000u >> __clz(e));
+            g |= e;
+            carry_tie += tot;
+        }
+        uint32_t tot;
+        const uint32_t cs = __popc(g);
+        uint32_t off = carry_sel + group_scan_incl<G>(cs, sc.redu, &tot, gtid) - cs;
+        while (g) {
+            const int bit = __ffs(g) - 1;
+            if (off < (uint32_t)k_eff) sc.i2[off] = (wi << 5) + bit;
+            ++off;
+            g &= g - 1;
+        }
+        carry_sel += tot;
+    }
+    G::sync();
+    // alpha = approximate-score mass of the selected set (Step 3)
+    float apart = 0.f;
+    for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[sc.i2[j]]) - vmax) * c1);
+    const float alpha = group_sum<G>(apart, sc.red, gtid) / Z;
+
+    // -------------------------------------------------------------- a5: gather k rows of K and V
+    const int hw = gtid >> 4, l16 = gtid & 15;
+    const float qscale = rsqrtf((float)D) * LOG2E;
+    float qs[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qs[e] = hm.qf[l16 * 8 + e] * qscale;
+    const uint4* Kh = reinterpret_cast<const uint4*>(K_head);
+    const uint4* Vh = reinterpret_cast<const uint4*>(V_head);
+    float m = -CUDART_INF_F, l = 0.f, acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int jb = 0; jb < k_eff; jb += G::NHW * RG) {        // trip count uniform across the group
+        uint4 kv[RG], vv[RG];
+#pragma unroll
+        for (int u = 0; u < RG; ++u) {
+            const int t = sc.i2[min(jb + u * G::NHW + hw, k_eff - 1)];
+            kv[u] = ld_stream(Kh + (size_t)t * (D / 8) + l16);
+            vv[u] = ld_stream(Vh + (size_t)t * (D / 8) + l16);
+        }
+        float z[RG], bmax = -CUDART_INF_F;
+#pragma unroll
+        for (int u = 0; u < RG; ++u) {
+            const __half2* kh = reinterpret_cast<const __half2*>(&kv[u]);
+            float zz = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 f = __half22float2(kh[e]);
+                zz = fmaf(f.x, qs[2 * e], zz);
+                zz = fmaf(f.y, qs[2 * e + 1], zz);
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) zz += __shfl_xor_sync(FULL, zz, o);
+            z[u] = (jb + u * G::NHW + hw < k_eff) ? zz : -CUDART_INF_F;   // uniform within the half-warp
+            bmax = fmaxf(bmax, z[u]);
+        }
+        const float mn = fmaxf(m, bmax);
+        if (mn > -CUDART_INF_F) {
+            const float scl = ex2(m - mn);
+            l *= scl;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] *= scl;
+#pragma unroll
+            for (int u = 0; u < RG; ++u) {
+                const float p = ex2(z[u] - mn);
+                l += p;
+                const __half2* vh = reinterpret_cast<const __half2*>(&vv[u]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(vh[e]);
+                    acc[2 * e] = fmaf(p, f.x, acc[2 * e]);
+                    acc[2 * e + 1] = fmaf(p, f.y, acc[2 * e + 1]);
+                }
+            }
+            m = mn;
+        }
+    }
+    // merge the half-warps' partial softmax states
+    float* mg = sc.merge + hw * (D + 2);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mg[l16 * 8 + e] = acc[e];
+    if (l16 == 0) { mg[D] = m; mg[D + 1] = l; }
+    G::sync();
+
+    // -------------------------------------------------------------- a6: combine with v_bar
+    if (gtid < D) {
+        const float vb = __half2float(__ushort_as_half(vbar_head[gtid]));
+        float M = -CUDART_INF_F;
+#pragma unroll
+        for (int w = 0; w < G::NHW; ++w) M = fmaxf(M, sc.merge[w * (D + 2) + D]);
+        float L = 0.f, s = 0.f;
+#pragma unroll
+        for (int w = 0; w < G::NHW; ++w) {
+            const float scl = ex2(sc.merge[w * (D + 2) + D] - M);
+            L = fmaf(sc.merge[w * (D + 2) + D + 1], scl, L);
+            s = fmaf(sc.merge[w * (D + 2) + gtid], scl, s);
+        }
+        out_row[gtid] = __half_as_ushort(__float2half_rn(alpha * (s / L) + (1.f - alpha) * vb));
+    }
+    if (gtid == 0 && alpha_out) *alpha_out = alpha;
+    if (idx_k_row) for (int j = gtid; j < k; j += G::NT) idx_k_row[j] = (j < k_eff) ? sc.i2[j] : -1;
+}
+
+}  // namespace sparq

@@ -1,0 +1,326 @@
+// sparq_decode, persistent warp-specialised kernel: one CTA per SM walks over (batch, query head)
+// units, and the three kinds of work of a unit run on different warps so that the HBM stream
+// never waits for the latency-bound stages:
+//
+//   producer warp     a1 for the NEXT unit (top-r of |q|, tau) while the current one streams, then
+//                     the bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast) of the
+//                     r selected Kt rows into a ring of shared-memory stages; lanes issue one row each
+//   stream group      a2: consumes the ring, fp32 mixed-precision FMA chain per position, writes the
+//                     order-preserving keys of unit j into key buffer j mod 3
+//   post groups 0/1   a3-a6 of units j = 0,2,4,.. / 1,3,5,.. (decode_common.cuh): radix select with
+//                     exact re-decision of the threshold band, alpha, K/V row gather, combine
+//
+// Hand-offs are mbarriers (ring full/empty, unit metadata full/free, key buffer full/free); every
+// wait is bounded: a wait that gives up raises SPARQ_DEV_TIMEOUT and sets a CTA-wide flag after
+// which no wait blocks any more, so the kernel always terminates.
+#include "decode_common.cuh"
+#include "kernels.h"
+
+namespace sparq {
+namespace {
+
+constexpr int SNT = 256;                 // stream-group threads
+constexpr int GNT = 256;                 // threads of one post group
+constexpr int NPOST = 2;
+constexpr int NT = 32 + SNT + NPOST * GNT;
+constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
+constexpr int RB = 8;                    // Kt rows per ring stage
+constexpr int STAGES = 3;
+constexpr int STAGE_BYTES = RB * CH * 2;
+constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+constexpr int NKB = 3;                   // key buffers: one being written, two being post-processed
+constexpr int NMETA = 4;                 // unit metadata slots in flight
+using SG = Group<SNT, 1>;
+using PG0 = Group<GNT, 2>;
+using PG1 = Group<GNT, 3>;
+static_assert(RB <= 8, "HeadMeta::qh padding");
+
+struct PipeShared {
+    HeadMeta meta[NMETA];
+    int32_t i2[NPOST][SPARQ_K_MAX];
+    uint64_t full[STAGES], empty[STAGES];          // ring stage landed / consumed
+    uint64_t meta_full[NMETA], meta_free[NMETA];   // a1 done / unit finished
+    uint64_t keys_full[NKB], keys_free[NKB];       // keys of a unit complete / post-processed
+    uint32_t kmax[NKB];
+    float kabs[NKB];
+    float red[NPOST][2 * (GNT / 32)];
+    uint32_t redu[NPOST][2 * (GNT / 32)];
+    uint32_t res[NPOST][4];
+    uint32_t band[NPOST][4];
+    uint32_t sredu[2 * (SNT / 32)];
+    int abort_flag;
+};
+
+struct Args {
+    const sparq_half *q, *K, *Kt, *V, *vbar;
+    const int32_t* seq_lens;
+    int n_units, Hq, Hkv, S_max, S_cap, r, k;
+    sparq_half* out;
+    int32_t *idx_r, *idx_k;
+    float* alpha;
+    int32_t* status;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Bounded wait.  Gives up after WAIT_LIMIT polls, or at once when another thread already gave up.
+__device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, PipeShared& sh, int32_t* status) {
+    volatile int* flag = &sh.abort_flag;
+    for (int i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((i & 63) == 63 && *flag) return;
+    }
+    *flag = 1;
+    raise_status(status, SPARQ_DEV_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------------- producer
+__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine) {
+    const int lane = threadIdx.x & 31;
+    const int g_heads = a.Hq / a.Hkv;
+    uint32_t g = 0;                                          // ring stages issued so far
+    uint2 qraw = make_uint2(0, 0);                           // components 4*lane .. 4*lane+3 of the unit's q
+    if (n_mine > 0) qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)blockIdx.x * D + lane * 4);
+    for (int j = 0; j < n_mine; ++j) {
+        const int bh = blockIdx.x + j * gridDim.x, b = bh / a.Hq, h = bh % a.Hq;
+        const int m = j % NMETA;
+        HeadMeta& hm = sh.meta[m];
+        wait_or_abort(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
+
+        // ---- a1: top-r of |q| for this unit; key = |q_c| bits above (127 - c)
+        const int n = a.seq_lens[b];
+        const bool valid = n >= 1 && n <= a.S_max;
+        const int k_eff = valid ? min(a.k, n) : 0;
+        const uint16_t hb[4] = {(uint16_t)(qraw.x & 0xffffu), (uint16_t)(qraw.x >> 16), (uint16_t)(qraw.y & 0xffffu),
+                                (uint16_t)(qraw.y >> 16)};
+        float qf[4], l1_all = 0.f;
+        uint32_t mine[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int c = lane * 4 + e;
+            qf[e] = __half2float(__ushort_as_half(hb[e]));
+            l1_all += fabsf(qf[e]);
+            mine[e] = ((uint32_t)(hb[e] & 0x7fffu) << 7) | (uint32_t)(D - 1 - c);
+            hm.qf[c] = qf[e];
+            hm.rkey[c] = mine[e];
+        }
+        __syncwarp();
+        int rank[4] = {0, 0, 0, 0};
+        const uint4* rk4 = reinterpret_cast<const uint4*>(hm.rkey);
+#pragma unroll 4
+        for (int i = 0; i < D / 4; ++i) {
+            const uint4 o = rk4[i];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) rank[e] += (o.x > mine[e]) + (o.y > mine[e]) + (o.z > mine[e]) + (o.w > mine[e]);
+        }
+        int cnt = 0;
+        float l1_sel = 0.f;
+        bool sel[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { sel[e] = rank[e] < a.r; cnt += sel[e]; l1_sel += sel[e] ? fabsf(qf[e]) : 0.f; }
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
+        int slot = incl - cnt;                               // ascending component order: by lane, then e
+#pragma unroll
+        for (int e = 0; e < 4; ++e) if (sel[e]) { hm.i1[slot] = lane * 4 + e; hm.qh[slot] = hb[e]; ++slot; }
+        l1_all = warp_sum(l1_all);
+        l1_sel = warp_sum(l1_sel);
+        const int r_pad = (a.r + RB - 1) / RB * RB;
+        for (int c = a.r + lane; c < r_pad; c += 32) hm.qh[c] = 0;
+        if (lane == 0) {
+            hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = valid;
+            hm.inv_tau = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
+            hm.l1_sel = l1_sel;
+        }
+        __syncwarp();
+        if (a.idx_r) for (int c = lane; c < a.r; c += 32) a.idx_r[(size_t)bh * a.r + c] = valid ? hm.i1[c] : -1;
+        // the next unit's query travels while this unit's rows are issued
+        if (j + 1 < n_mine) qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)(bh + gridDim.x) * D + lane * 4);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.meta_full[m]);
+
+        // ---- issue the unit's ring stages: [chunk c][row batch jb] -> RB rows x CH positions
+        if (k_eff > 0) {
+            const sparq_half* Kt_head = a.Kt + ((size_t)b * a.Hkv + h / g_heads) * (size_t)D * a.S_max;
+            const int n8 = (n + 7) & ~7;
+            const int n_chunks = (n8 + CH - 1) / CH;
+            for (int c = 0; c < n_chunks; ++c) {
+                const uint32_t bytes = (uint32_t)min(CH, n8 - c * CH) * 2u;
+                for (int jb = 0; jb < a.r; jb += RB, ++g) {
+                    const int s = g % STAGES;
+                    const int rows = min(RB, a.r - jb);
+                    wait_or_abort(&sh.empty[s], ((g / STAGES) & 1u) ^ 1u, sh, a.status);
+                    if (lane == 0) mbar_expect_tx(&sh.full[s], bytes * rows);
+                    __syncwarp();
+                    if (lane < rows)
+                        bulk_g2s(ring + s * STAGE_BYTES + lane * (CH * 2),
+                                 Kt_head + (size_t)hm.i1[jb + lane] * a.S_max + c * CH, bytes, &sh.full[s]);
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------- stream group
+__device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
+                                            int n_mine) {
+    const int gtid = threadIdx.x - 32, lane = gtid & 31;
+    uint32_t g = 0;
+    for (int j = 0; j < n_mine; ++j) {
+        const int m = j % NMETA, kb = j % NKB;
+        const HeadMeta& hm = sh.meta[m];
+        uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
+        wait_or_abort(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        wait_or_abort(&sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
+        const int n = hm.n, r = a.r;
+        if (hm.k_eff > 0) {
+            uint32_t kmax = 0;
+            __half2 mx[4];                                   // largest |K| among the valid streamed values
+#pragma unroll
+            for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
+            const int n8 = (n + 7) & ~7;
+            const int n_chunks = (n8 + CH - 1) / CH;
+            for (int c = 0; c < n_chunks; ++c) {
+                float acc[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                const int t0 = c * CH + gtid * 8;
+                const int nvalid = min(8, n - t0);           // positions of this thread's vector inside the sequence
+                // positions past n in the straddling vector hold whatever the caller's memory holds: mask them
+                uint32_t msk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
+                for (int jb = 0; jb < r; jb += RB, ++g) {
+                    const int s = g % STAGES;
+                    wait_or_abort(&sh.full[s], (g / STAGES) & 1u, sh, a.status);
+                    const uint4* src = reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid;
+                    if (nvalid >= 8) {
+#pragma unroll
+                        for (int u = 0; u < RB; ++u)
+                            if (jb + u < r) row_fma(acc, mx, src[u * (CH / 8)], hm.qh[jb + u]);   // uniform; padded rows were not copied
+                    } else if (nvalid > 0) {
+#pragma unroll
+                        for (int u = 0; u < RB; ++u)
+                            if (jb + u < r) {
+                                uint4 v = src[u * (CH / 8)];
+                                v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
+                                row_fma(acc, mx, v, hm.qh[jb + u]);
+                            }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.empty[s]);   // this warp is done with slot s
+                }
+                uint32_t kk[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) kk[e] = key32(acc[e]);
+                if (nvalid >= 8) {
+                    *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+                    *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) kmax = max(kmax, kk[e]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) if (e < nvalid) { keys[t0 + e] = kk[e]; kmax = max(kmax, kk[e]); }
+                }
+            }
+            uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
+            group_max2_u32<SG>(kmax, kabs_bits, sh.sredu, gtid);
+            if (gtid == 0) { sh.kmax[kb] = kmax; sh.kabs[kb] = __uint_as_float(kabs_bits); }
+        }
+        SG::sync();                                          // every key of the unit is written
+        if (gtid == 0) mbar_arrive(&sh.keys_full[kb]);
+    }
+}
+
+// ---------------------------------------------------------------------------------- post groups
+template <class PG>
+__device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, unsigned char* scratch,
+                                          int n_mine, int p) {
+    const int gtid = threadIdx.x - 32 - SNT - p * GNT;
+    PostScratch sc;
+    carve_post_scratch(sc, scratch, PG::NHW, a.S_cap / 32);
+    sc.i2 = sh.i2[p]; sc.red = sh.red[p]; sc.redu = sh.redu[p]; sc.res = sh.res[p]; sc.band = sh.band[p];
+    const int g_heads = a.Hq / a.Hkv;
+    for (int j = p; j < n_mine; j += NPOST) {
+        const int m = j % NMETA, kb = j % NKB;
+        const HeadMeta& hm = sh.meta[m];
+        wait_or_abort(&sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
+        const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq;
+        const size_t kv_head = (size_t)b * a.Hkv + h / g_heads;
+        sparq_half* out_row = a.out + (size_t)bh * D;
+        if (!hm.valid) {                                     // defined result, no trap
+            if (gtid == 0) { raise_status(a.status, SPARQ_DEV_BAD_SEQ_LEN); if (a.alpha) a.alpha[bh] = 0.f; }
+            if (gtid < D) out_row[gtid] = 0;
+            if (a.idx_k) for (int i = gtid; i < a.k; i += GNT) a.idx_k[(size_t)bh * a.k + i] = -1;
+        } else if (hm.k_eff == 0) {                          // nothing to select: the mean value vector
+            if (gtid < D) out_row[gtid] = a.vbar[kv_head * D + gtid];
+            if (gtid == 0 && a.alpha) a.alpha[bh] = 0.f;
+        } else {
+            post_phase<PG>(gtid, hm, keys_all + (size_t)kb * a.S_cap, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.k, a.S_max,
+                           a.Kt + kv_head * (size_t)D * a.S_max, a.K + kv_head * (size_t)a.S_max * D,
+                           a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
+                           a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
+        }
+        PG::sync();                                          // the group is done with the keys, the metadata, i2
+        if (gtid == 0) { mbar_arrive(&sh.keys_free[kb]); mbar_arrive(&sh.meta_free[m]); }
+    }
+}
+
+__global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    unsigned char* ring = dyn_smem;
+    uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);
+    unsigned char* scratch0 = dyn_smem + RING_BYTES + (size_t)NKB * a.S_cap * 4;
+    const size_t scratch_bytes = (post_scratch_bytes(GNT / 16, a.S_cap / 32) + 127) & ~(size_t)127;
+    __shared__ PipeShared sh;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], SNT / 32); }
+        for (int m = 0; m < NMETA; ++m) { mbar_init(&sh.meta_full[m], 1); mbar_init(&sh.meta_free[m], 1); }
+        for (int b = 0; b < NKB; ++b) { mbar_init(&sh.keys_full[b], 1); mbar_init(&sh.keys_free[b], 1); }
+        sh.abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const int n_mine = (a.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units blockIdx.x + j*gridDim.x
+    const int warp = threadIdx.x >> 5;
+    if (warp == 0) producer_role(a, sh, ring, n_mine);
+    else if (warp <= SNT / 32) stream_role(a, sh, ring, keys_all, n_mine);
+    else if (warp <= SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, scratch0, n_mine, 0);
+    else post_role<PG1>(a, sh, keys_all, scratch0 + scratch_bytes, n_mine, 1);
+}
+
+size_t pipe_dynamic_smem(int S_cap) {
+    const size_t scratch = (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127;
+    return (size_t)RING_BYTES + (size_t)NKB * S_cap * 4 + NPOST * scratch;
+}
+
+}  // namespace
+
+// S_max rounded up so that bitmap words and 16-byte key vectors stay whole
+static int pipe_s_cap(int S_max) { return (S_max + 127) & ~127; }
+
+bool pipe_fits(int S_max, int smem_optin) {
+    return pipe_dynamic_smem(pipe_s_cap(S_max)) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
+}
+
+cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                                     const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
+                                     int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                     int32_t* status, int n_sm, cudaStream_t stream) {
+    Args a;
+    a.q = q; a.K = K; a.Kt = Kt; a.V = V; a.vbar = vbar; a.seq_lens = seq_lens;
+    a.n_units = B * Hq; a.Hq = Hq; a.Hkv = Hkv; a.S_max = S_max; a.S_cap = pipe_s_cap(S_max); a.r = r; a.k = k;
+    a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status;
+    const size_t dyn = pipe_dynamic_smem(a.S_cap);
+    cudaError_t e = cudaFuncSetAttribute(sparq_decode_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    if (e != cudaSuccess) return e;
+    const int grid = a.n_units < n_sm ? a.n_units : n_sm;
+    sparq_decode_pipe_kernel<<<grid, NT, dyn, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace sparq
