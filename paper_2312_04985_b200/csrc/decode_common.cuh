@@ -24,7 +24,7 @@ struct Group {
 };
 
 // What the later stages need to know about one (batch, query head) unit; filled by stage a1.
-struct HeadMeta {
+struct alignas(16) HeadMeta {
     float qf[D];                  // q as fp32
     int32_t i1[D];                // selected components, ascending
     uint32_t rkey[D];             // a1 scratch: ranking keys
@@ -362,7 +362,8 @@ __device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const u
         uint4 kv[RG], vv[RG];
 #pragma unroll
         for (int u = 0; u < RG; ++u) {
-            const int t = sc.i2[min(jb + u * G::NHW + hw, k_eff - 1)];
+            // (the clamp keeps the address inside the head even if the list were ever corrupt)
+            const int t = min(max(sc.i2[min(jb + u * G::NHW + hw, k_eff - 1)], 0), n - 1);
             kv[u] = ld_stream(Kh + (size_t)t * (D / 8) + l16);
             vv[u] = ld_stream(Vh + (size_t)t * (D / 8) + l16);
         }

@@ -35,6 +35,18 @@ using PG0 = Group<GNT, 2>;
 using PG1 = Group<GNT, 3>;
 static_assert(RB <= 8, "HeadMeta::qh padding");
 
+// Optional cycle counters for tuning (-DSPARQ_PHASE_CLOCKS): [0] post phase, [1] post waiting for keys,
+// [2] stream waiting for a free key buffer, [3] stream waiting for ring data, [4] stream total per unit,
+// [5] producer waiting for a free ring slot, [6] producer a1
+#ifdef SPARQ_PHASE_CLOCKS
+__device__ unsigned long long g_pipe_clocks[16];
+#define CLK_BEGIN(var) long long var = clock64()
+#define CLK_ADD(i, var, cond) do { if (cond) atomicAdd(&g_pipe_clocks[i], (unsigned long long)(clock64() - var)); } while (0)
+#else
+#define CLK_BEGIN(var)
+#define CLK_ADD(i, var, cond)
+#endif
+
 struct PipeShared {
     HeadMeta meta[NMETA];
     int32_t i2[NPOST][SPARQ_K_MAX];
@@ -88,6 +100,7 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
         const int m = j % NMETA;
         HeadMeta& hm = sh.meta[m];
         wait_or_abort(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
+        CLK_BEGIN(t_a1);
 
         // ---- a1: top-r of |q| for this unit; key = |q_c| bits above (127 - c)
         const int n = a.seq_lens[b];
@@ -141,6 +154,7 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
         if (j + 1 < n_mine) qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)(bh + gridDim.x) * D + lane * 4);
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.meta_full[m]);
+        CLK_ADD(6, t_a1, lane == 0);
 
         // ---- issue the unit's ring stages: [chunk c][row batch jb] -> RB rows x CH positions
         if (k_eff > 0) {
@@ -152,7 +166,9 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
                 for (int jb = 0; jb < a.r; jb += RB, ++g) {
                     const int s = g % STAGES;
                     const int rows = min(RB, a.r - jb);
+                    CLK_BEGIN(t_e);
                     wait_or_abort(&sh.empty[s], ((g / STAGES) & 1u) ^ 1u, sh, a.status);
+                    CLK_ADD(5, t_e, lane == 0);
                     if (lane == 0) mbar_expect_tx(&sh.full[s], bytes * rows);
                     __syncwarp();
                     if (lane < rows)
@@ -173,8 +189,11 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
+        CLK_BEGIN(t_unit);
         wait_or_abort(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        CLK_BEGIN(t_kf);
         wait_or_abort(&sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
+        CLK_ADD(2, t_kf, gtid == 0);
         const int n = hm.n, r = a.r;
         if (hm.k_eff > 0) {
             uint32_t kmax = 0;
@@ -195,7 +214,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
                 for (int jb = 0; jb < r; jb += RB, ++g) {
                     const int s = g % STAGES;
+                    CLK_BEGIN(t_f);
                     wait_or_abort(&sh.full[s], (g / STAGES) & 1u, sh, a.status);
+                    CLK_ADD(3, t_f, gtid == 0);
                     const uint4* src = reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid;
                     if (nvalid >= 8) {
 #pragma unroll
@@ -232,6 +253,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         }
         SG::sync();                                          // every key of the unit is written
         if (gtid == 0) mbar_arrive(&sh.keys_full[kb]);
+        CLK_ADD(4, t_unit, gtid == 0);
     }
 }
 
@@ -247,7 +269,10 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
     for (int j = p; j < n_mine; j += NPOST) {
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
+        CLK_BEGIN(t_w);
         wait_or_abort(&sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
+        CLK_ADD(1, t_w, gtid == 0);
+        CLK_BEGIN(t_p);
         const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq;
         const size_t kv_head = (size_t)b * a.Hkv + h / g_heads;
         sparq_half* out_row = a.out + (size_t)bh * D;
@@ -265,6 +290,7 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
                            a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
         }
         PG::sync();                                          // the group is done with the keys, the metadata, i2
+        CLK_ADD(0, t_p, gtid == 0);
         if (gtid == 0) { mbar_arrive(&sh.keys_free[kb]); mbar_arrive(&sh.meta_free[m]); }
     }
 }
@@ -299,6 +325,15 @@ size_t pipe_dynamic_smem(int S_cap) {
 }
 
 }  // namespace
+
+#ifdef SPARQ_PHASE_CLOCKS
+extern "C" int sparq_debug_pipe_clocks(unsigned long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    if (out16 && cudaMemcpyFromSymbol(out16, g_pipe_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_pipe_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+#endif
 
 // S_max rounded up so that bitmap words and 16-byte key vectors stay whole
 static int pipe_s_cap(int S_max) { return (S_max + 127) & ~127; }

@@ -58,6 +58,16 @@ def test_shrunk_batch_all_heads(name, kw):
     assert waived <= max(1, total // 200)
 
 
+def test_more_units_than_sms_all_heads():
+    """More (batch, head) units than SMs, so the persistent kernel's CTAs each walk several units
+    (ring, key-buffer and metadata slots wrap around) with ragged lengths and an invalid sequence."""
+    c = synth.make_case("c2", device="cuda", B=21, S=1024, ragged=(700, 1023))       # 672 units
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    waived, total = H.run_case_all_heads(c, "many units")
+    assert total == 672 and waived <= 3
+
+
 def test_dense_decode_on_workloads():
     for name, kw in (("c1", {}), ("c3", dict(B=2, S=5000, backend="numpy")),
                      ("c4", dict(B=3, n_steps=1, ragged=(700, 2500), backend="numpy"))):
