@@ -9,7 +9,6 @@ namespace sparq {
 
 constexpr int HIST_BINS = 2048;
 constexpr int CAND_MAX = 256;            // threshold-band positions the quick fp64 re-decision handles
-constexpr int RG = 8;                    // gathered rows in flight per half-warp
 constexpr int WAIT_LIMIT = 1 << 22;      // polls before an asynchronous copy is declared lost
 
 // A group of NT_ consecutive threads (whole warps) that synchronises on its own barrier.
@@ -87,6 +86,35 @@ __device__ __forceinline__ float mx_to_float(const __half2 (&mx)[4]) {
     return fmaxf(__low2float(a), __high2float(a));
 }
 
+// One ring stage (RB rows of CH8 16-byte vectors each) into a thread's 8 running sums.
+//   src: the thread's vector in row 0 of the stage; qh_jb: the RB query components of these rows
+//   (16-byte aligned); rows_left: selected rows not yet consumed (>= 1); nvalid: how many of the
+//   thread's 8 positions lie inside the sequence.
+// Positions past the sequence end in the straddling vector hold whatever the caller's memory
+// holds; they are masked to zero so that they reach neither a sum nor the |K| maximum.
+template <int RB, int CH8>
+__device__ __forceinline__ void stage_fma(float (&acc)[8], __half2 (&mx)[4], const uint4* src, const uint16_t* qh_jb,
+                                          int rows_left, int nvalid) {
+    static_assert(RB == 4 || RB == 8, "query components are fetched as one 8- or 16-byte vector");
+    if (nvalid >= 8 && rows_left >= RB) {                    // the common case: no predicates at all
+        uint32_t qw[RB / 2];
+        if constexpr (RB == 8) { const uint4 q8 = *reinterpret_cast<const uint4*>(qh_jb); qw[0] = q8.x; qw[1] = q8.y; qw[2] = q8.z; qw[3] = q8.w; }
+        else { const uint2 q4 = *reinterpret_cast<const uint2*>(qh_jb); qw[0] = q4.x; qw[1] = q4.y; }
+#pragma unroll
+        for (int u = 0; u < RB; ++u)
+            row_fma(acc, mx, src[u * CH8], (uint16_t)((u & 1) ? (qw[u >> 1] >> 16) : (qw[u >> 1] & 0xffffu)));
+    } else if (nvalid > 0) {
+        uint32_t msk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
+        for (int u = 0; u < RB && u < rows_left; ++u) {      // padded rows were not copied
+            uint4 v = src[u * CH8];
+            v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
+            row_fma(acc, mx, v, qh_jb[u]);
+        }
+    }
+}
+
 // ---- group-wide reductions in a fixed order (bitwise reproducible run to run) -------------
 template <class G>
 __device__ __forceinline__ float group_sum(float v, float* red, int gtid) {
@@ -143,11 +171,11 @@ __device__ __forceinline__ uint32_t group_scan_incl(uint32_t v, uint32_t* red, u
 // One radix-select pass over an already filled histogram: find, from the top, the bin holding the
 // need-th largest candidate.  res[0] = bin, res[1] = candidates above it, res[2] = candidates in
 // it.  All threads of the group call; the result is valid after the trailing barrier.
-template <class G>
+template <class G, int NBINS>
 __device__ __forceinline__ void find_bin(const uint32_t* hist, uint32_t need, uint32_t* red, uint32_t* res, int gtid) {
-    constexpr int PER = HIST_BINS / G::NT;
-    static_assert(HIST_BINS % G::NT == 0, "bins per thread");
-    const int top = HIST_BINS - 1 - gtid * PER;              // this thread's bins: top, top-1, ...
+    constexpr int PER = NBINS / G::NT;
+    static_assert(NBINS % G::NT == 0 && PER >= 1, "bins per thread");
+    const int top = NBINS - 1 - gtid * PER;                  // this thread's bins: top, top-1, ...
     uint32_t c[PER], s = 0;
 #pragma unroll
     for (int i = 0; i < PER; ++i) { c[i] = hist[top - i]; s += c[i]; }
@@ -180,24 +208,53 @@ __device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const Head
     return acc;
 }
 
-// Stages a4, a3, a5, a6 for one head, run by the thread group G (gtid = thread index in the group).
-//   keys[0..n): order-preserving keys of the fp32 approximate-score sums; kmax their maximum;
-//   kabs: largest |K| among the streamed values (error bound of the sums).
-// Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
-// group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
+// What a select variant hands to finish(): the selection bitmap sc.bm_sel (and, in the degenerate
+// path, the tie bitmap sc.bm_tie with need_tie of its lowest positions wanted) and the softmax
+// denominator of the approximate scores relative to the largest key.
+struct SelectResult {
+    float Z;
+    uint32_t need_tie;
+};
+
+// |fp32 chain - exact sum| <= ((1+u)^r - 1) sum_j |q_j K_tj| <= 1.02 r u ||q[i1]||_1 max|K|,  u = 2^-24
+__device__ __forceinline__ float two_b(int r, float l1_sel, float kabs) {
+    return 2.f * (1.02f * (float)r * 5.9604645e-8f * l1_sel * kabs);
+}
+
+// Re-decide the positions listed in sc.cand_pos[0..n_cand) (all keys within 2B of the threshold) by
+// their fp64 sums of exact products: the need64 largest (ties to the lowest position) get their
+// bitmap bit set, the others cleared.  n_cand <= CAND_MAX <= group size.
 template <class G>
-__device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, float kabs,
-                                           const PostScratch& sc, int r, int k, int S_max,
-                                           const sparq_half* __restrict__ Kt_head, const sparq_half* __restrict__ K_head,
-                                           const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
-                                           sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
-                                           float* __restrict__ alpha_out) {
+__device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, const PostScratch& sc, uint32_t n_cand,
+                                              uint32_t need64, const sparq_half* Kt_head, int S_max, int r) {
+    static_assert(CAND_MAX <= G::NT, "one thread per band candidate");
+    unsigned long long v = 0;
+    int t = 0;
+    if (gtid < n_cand) { t = sc.cand_pos[gtid]; v = key64(dot64_at(Kt_head, hm, S_max, r, t)); sc.cand_val[gtid] = v; }
+    G::sync();
+    if (gtid < n_cand) {
+        uint32_t rank = 0;
+        for (uint32_t i = 0; i < n_cand; ++i) {
+            const unsigned long long vi = sc.cand_val[i];
+            rank += (vi > v) || (vi == v && sc.cand_pos[i] < t);
+        }
+        if (rank < need64) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
+        else atomicAnd(&sc.bm_sel[t >> 5], ~(1u << (t & 31)));
+    }
+    G::sync();
+}
+
+// Stages a4 + a3 from the keys alone (any n): MSB radix select over all keys, 11 + 11 + 10 bits,
+// then one pass for the softmax denominator, the bitmap and the threshold band.
+template <class G>
+__device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+                                                       float kabs, const PostScratch& sc, int r, int S_max,
+                                                       const sparq_half* __restrict__ Kt_head) {
     const int lane = gtid & 31, warp = gtid >> 5;
     const int n = hm.n, k_eff = hm.k_eff;
     const float inv_tau = hm.inv_tau;
     const float vmax = unkey32(kmax);
-    // |fp32 chain - exact sum| <= ((1+u)^r - 1) sum_j |q_j K_tj| <= 1.02 r u ||q[i1]||_1 max|K|,  u = 2^-24
-    const float twoB = 2.f * (1.02f * (float)r * 5.9604645e-8f * hm.l1_sel * kabs);
+    const float twoB = two_b(r, hm.l1_sel, kabs);
 
     // -------------------------------------------------------------- a4: top-k select
     // MSB radix select, 11 + 11 + 10 bits, leaving the loop as soon as a whole bin is wanted.
@@ -217,7 +274,7 @@ __device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const u
                 if ((u & mask) == prefix) atomicAdd(&sc.hist[(u >> shift) & ((1u << bits) - 1)], 1u);
             }
             G::sync();
-            find_bin<G>(sc.hist, need, sc.redu, sc.res, gtid);
+            find_bin<G, HIST_BINS>(sc.hist, need, sc.redu, sc.res, gtid);
             prefix |= sc.res[0] << shift;
             mask |= ((1u << bits) - 1) << shift;
             need -= sc.res[1];
@@ -261,22 +318,7 @@ __device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const u
         // sums of exact products; equal fp64 sums go to the lowest positions.
         const uint32_t need64 = cnt_hi - over;
         if (n_cand <= CAND_MAX) {
-            // few candidates: one thread each, rank by counting, then patch their bitmap bits
-            static_assert(CAND_MAX <= G::NT, "one thread per band candidate");
-            unsigned long long v = 0;
-            int t = 0;
-            if (gtid < n_cand) { t = sc.cand_pos[gtid]; v = key64(dot64_at(Kt_head, hm, S_max, r, t)); sc.cand_val[gtid] = v; }
-            G::sync();
-            if (gtid < n_cand) {
-                uint32_t rank = 0;
-                for (uint32_t i = 0; i < n_cand; ++i) {
-                    const unsigned long long vi = sc.cand_val[i];
-                    rank += (vi > v) || (vi == v && sc.cand_pos[i] < t);
-                }
-                if (rank < need64) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
-                else atomicAnd(&sc.bm_sel[t >> 5], ~(1u << (t & 31)));
-            }
-            G::sync();
+            redecide_band<G>(gtid, hm, sc, n_cand, need64, Kt_head, S_max, r);
         } else {
             // many candidates (degenerate inputs, e.g. constant keys): radix select over their
             // 64-bit keys, 8 passes of 8 bits, then rebuild the bitmap
@@ -294,7 +336,7 @@ __device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const u
                     }
                 }
                 G::sync();
-                find_bin<G>(sc.hist, left, sc.redu, sc.res, gtid);
+                find_bin<G, HIST_BINS>(sc.hist, left, sc.redu, sc.res, gtid);
                 p64 |= (unsigned long long)sc.res[0] << shift;
                 m64 |= 255ull << shift;
                 left -= sc.res[1];
@@ -315,6 +357,141 @@ __device__ __forceinline__ void post_phase(int gtid, const HeadMeta& hm, const u
             G::sync();
         }
     }
+
+    SelectResult res;
+    res.Z = Z;
+    res.need_tie = need_tie;
+    return res;
+}
+
+// First-digit histogram the stream stage fills while the keys are still in registers.
+constexpr int FB = 10, FSH = 32 - FB, FBINS = 1 << FB;
+constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the threshold bin; the list lives in sc.hist
+
+// Stages a4 + a3 when hist1 already holds the histogram of the keys' top FB bits.  One scan of the
+// keys builds the bitmap of everything above the threshold bin, the softmax denominator and the list
+// of the bin's own keys; the threshold is then resolved inside that short list, and the 2B band
+// around it re-decided in fp64 as in select_generic.  Clears hist1 for its next user.
+// Returns false (for every thread of the group alike) when the short-cut does not apply -- the bin
+// holds more keys than the list, or the band reaches outside the bin or holds too many keys -- and
+// the caller runs select_generic instead.
+template <class G>
+__device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+                                                 float kabs, const PostScratch& sc, uint32_t* hist1, int r, int S_max,
+                                                 const sparq_half* __restrict__ Kt_head, SelectResult& out) {
+    static_assert(G::NT >= 256, "warp 0 scans 256 bins, thread i clears bin i");
+    const int lane = gtid & 31, warp = gtid >> 5;
+    const int n = hm.n, k_eff = hm.k_eff;
+    const float vmax = unkey32(kmax);
+    const float c1 = hm.inv_tau * LOG2E;
+
+    if (gtid < 4) sc.band[gtid] = 0;     // [0] band keys below the edge, [1] at/above it, [2] band list, [3] bin list
+    find_bin<G, FBINS>(hist1, (uint32_t)k_eff, sc.redu, sc.res, gtid);
+    const uint32_t b1 = sc.res[0], above = sc.res[1];
+    for (int i = gtid; i < FBINS / 4; i += G::NT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
+    uint32_t* list_key = sc.hist;
+    int32_t* list_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX);
+
+    const int nwords = (n + 31) >> 5;
+    float zpart = 0.f;
+    for (int wi = warp; wi < nwords; wi += G::NW) {
+        const int t = (wi << 5) + lane;
+        const bool valid = t < n;
+        const uint32_t u = valid ? keys[t] : 0u;
+        zpart += valid ? ex2((unkey32(u) - vmax) * c1) : 0.f;
+        const uint32_t dig = u >> FSH;
+        const unsigned g = __ballot_sync(FULL, valid && dig > b1);
+        if (lane == 0) sc.bm_sel[wi] = g;
+        if (valid && dig == b1) {
+            const uint32_t slot = atomicAdd(&sc.band[3], 1u);
+            if (slot < LIST_MAX) { list_key[slot] = u; list_pos[slot] = t; }
+        }
+    }
+    out.Z = group_sum<G>(zpart, sc.red, gtid);               // barriers also publish the bitmap and the list
+    out.need_tie = 0;
+    const uint32_t m = sc.band[3];
+    if (m > LIST_MAX) return false;
+
+    // the threshold among the bin's m keys: `need` of them are wanted; remaining 22 bits as 8 + 8 + 6
+    uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH, mask = ~0u << FSH, ceq = m;
+    uint32_t* h256 = reinterpret_cast<uint32_t*>(sc.cand_val);
+    int shift = FSH;
+#pragma unroll 1
+    for (int pass = 0; pass < 3 && ceq != need; ++pass) {
+        const int bits = pass < 2 ? 8 : 6;
+        shift -= bits;
+        if (gtid < 256) h256[gtid] = 0;
+        G::sync();
+        for (uint32_t i = gtid; i < m; i += G::NT) {
+            const uint32_t u = list_key[i];
+            if ((u & mask) == prefix) atomicAdd(&h256[(u >> shift) & ((1u << bits) - 1)], 1u);
+        }
+        G::sync();
+        if (warp == 0) {                                     // 8 bins per lane, from the top
+            uint32_t c[8], sum = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = h256[255 - (lane * 8 + i)]; sum += c[i]; }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
+            uint32_t run = incl - sum;
+            if (run < need && need <= incl) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (run + c[i] >= need) { sc.res[0] = 255 - (lane * 8 + i); sc.res[1] = run; sc.res[2] = c[i]; break; }
+                    run += c[i];
+                }
+            }
+        }
+        G::sync();
+        prefix |= sc.res[0] << shift;
+        mask |= ((1u << bits) - 1) << shift;
+        need -= sc.res[1];
+        ceq = sc.res[2];
+    }
+    const uint32_t edge = prefix;                            // unprocessed low bits are zero
+    const uint32_t over = ceq - need;
+    const float twoB = two_b(r, hm.l1_sel, kabs);
+    const float edge_val = unkey32(edge);
+    const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
+    if ((lo_key >> FSH) != b1 || (hi_key >> FSH) != b1) return false;   // keys outside the list may be in the band
+
+    for (uint32_t i = gtid; i < m; i += G::NT) {
+        const uint32_t u = list_key[i];
+        const int t = list_pos[i];
+        if (u >= edge) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
+        if (u >= lo_key && u <= hi_key) {
+            atomicAdd(&sc.band[u >= edge ? 1 : 0], 1u);
+            const uint32_t slot = atomicAdd(&sc.band[2], 1u);
+            if (slot < CAND_MAX) sc.cand_pos[slot] = t;
+        }
+    }
+    G::sync();
+    const uint32_t cnt_lo = sc.band[0], cnt_hi = sc.band[1], n_cand = sc.band[2];
+    if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
+        if (n_cand > CAND_MAX) return false;
+        redecide_band<G>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
+    }
+    return true;
+}
+
+// Stages a5 and a6 for one unit from a finished selection: ascending index list from the bitmap(s),
+// alpha, gather of the selected K and V rows with online softmax, combine with v_bar.
+// RG: gathered K and V rows in flight per half-warp (register budget of the calling kernel).
+// Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
+// group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
+template <class G, int RG>
+__device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, SelectResult sel,
+                                       const PostScratch& sc, int k, const sparq_half* __restrict__ K_head,
+                                       const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
+                                       sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
+                                       float* __restrict__ alpha_out) {
+    const int n = hm.n, k_eff = hm.k_eff;
+    const int nwords = (n + 31) >> 5;
+    const float vmax = unkey32(kmax);
+    const float c1 = hm.inv_tau * LOG2E;
+    const float Z = sel.Z;
+    const uint32_t need_tie = sel.need_tie;
 
     // ascending list of selected positions from the bitmap(s)
     uint32_t carry_tie = 0, carry_sel = 0;

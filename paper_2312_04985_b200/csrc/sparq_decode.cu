@@ -29,6 +29,7 @@ using CTA = Group<NT, 0>;
 static_assert(post_scratch_bytes(CTA::NHW, BM_WORDS) <= RING_BYTES, "post-phase scratch must fit the dead ring");
 static_assert(RB <= 8, "HeadMeta::qh padding");
 
+
 // Optional per-phase cycle counters (thread 0 of every CTA, summed over CTAs); compiled in only
 // with -DSPARQ_PHASE_CLOCKS for tuning, never in the shipped library.
 #ifdef SPARQ_PHASE_CLOCKS
@@ -173,26 +174,9 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         const int t0 = c * CH + tid * 8;
         const int nvalid = min(8, n - t0);                   // positions of this thread's vector inside the sequence
-        // positions past n in the straddling vector hold whatever the caller's memory holds: mask them
-        uint32_t msk[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
         for (int jb = 0; jb < r_pad; jb += RB, ++it) {
             ok = mbar_wait_bounded(&sh.full[s], parity, WAIT_LIMIT);
-            const uint4* src = reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + tid;
-            if (nvalid >= 8) {
-#pragma unroll
-                for (int u = 0; u < RB; ++u)
-                    if (jb + u < r) row_fma(acc, mx, src[u * (CH / 8)], hm.qh[jb + u]);   // uniform; padded rows were not copied
-            } else if (nvalid > 0) {
-#pragma unroll
-                for (int u = 0; u < RB; ++u)
-                    if (jb + u < r) {
-                        uint4 v = src[u * (CH / 8)];
-                        v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
-                        row_fma(acc, mx, v, hm.qh[jb + u]);
-                    }
-            }
+            stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + tid, hm.qh + jb, r - jb, nvalid);
             ok = __syncthreads_and(ok);                      // slot s fully consumed (or a wait gave up)
             if (!ok) break;
             if (warp == 0 && it + STAGES < total) issue(it + STAGES, s);
@@ -226,9 +210,9 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     PostScratch sc;
     carve_post_scratch(sc, ring, CTA::NHW, BM_WORDS);
     sc.i2 = sh.i2; sc.red = sh.red; sc.redu = sh.redu; sc.res = sh.res; sc.band = sh.band;
-    post_phase<CTA>(tid, hm, keys, kmax, __uint_as_float(kabs_bits), sc, r, k, S_max, Kt_head,
-                    K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D, vbar + kv_head * D, out_row,
-                    idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
+    const SelectResult sel_res = select_generic<CTA>(tid, hm, keys, kmax, __uint_as_float(kabs_bits), sc, r, S_max, Kt_head);
+    finish<CTA, 8>(tid, hm, keys, kmax, sel_res, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
+                   vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
     PHASE_MARK(2);
 }
 

@@ -2,8 +2,8 @@
 // units, and the three kinds of work of a unit run on different warps so that the HBM stream
 // never waits for the latency-bound stages:
 //
-//   producer warp     a1 for the NEXT unit (top-r of |q|, tau) while the current one streams, then
-//                     the bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast) of the
+//   a1 warp           top-r of |q| and tau for the units ahead (metadata slots), off everyone's path
+//   producer warp     the bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast) of the
 //                     r selected Kt rows into a ring of shared-memory stages; lanes issue one row each
 //   stream group      a2: consumes the ring, fp32 mixed-precision FMA chain per position, writes the
 //                     order-preserving keys of unit j into key buffer j mod 3
@@ -22,7 +22,8 @@ namespace {
 constexpr int SNT = 256;                 // stream-group threads
 constexpr int GNT = 256;                 // threads of one post group
 constexpr int NPOST = 2;
-constexpr int NT = 32 + SNT + NPOST * GNT;
+constexpr int LEAD = 64;                 // producer warp + a1 warp
+constexpr int NT = LEAD + SNT + NPOST * GNT;
 constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
 constexpr int RB = 8;                    // Kt rows per ring stage
 constexpr int STAGES = 3;
@@ -77,37 +78,47 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// Bounded wait.  Gives up after WAIT_LIMIT polls, or at once when another thread already gave up.
+// Bounded wait.  Between polls the warp sleeps NS nanoseconds so that waiting warps leave the issue
+// slots to the working ones.  Gives up after WAIT_LIMIT polls, or at once when another thread
+// already gave up; from then on no wait in this CTA blocks.
+template <int NS>
 __device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, PipeShared& sh, int32_t* status) {
     volatile int* flag = &sh.abort_flag;
     for (int i = 0; i < WAIT_LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return;
         if ((i & 63) == 63 && *flag) return;
+        __nanosleep(NS);
     }
     *flag = 1;
     raise_status(status, SPARQ_DEV_TIMEOUT);
 }
 
-// ---------------------------------------------------------------------------------- producer
-__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine) {
+// ---------------------------------------------------------------------------------- a1 warp
+__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_mine) {
     const int lane = threadIdx.x & 31;
-    const int g_heads = a.Hq / a.Hkv;
-    uint32_t g = 0;                                          // ring stages issued so far
     uint2 qraw = make_uint2(0, 0);                           // components 4*lane .. 4*lane+3 of the unit's q
-    if (n_mine > 0) qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)blockIdx.x * D + lane * 4);
+    int n_next = 0;
+    if (n_mine > 0) {
+        qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)blockIdx.x * D + lane * 4);
+        n_next = a.seq_lens[blockIdx.x / a.Hq];
+    }
     for (int j = 0; j < n_mine; ++j) {
-        const int bh = blockIdx.x + j * gridDim.x, b = bh / a.Hq, h = bh % a.Hq;
+        const int bh = blockIdx.x + j * gridDim.x;
         const int m = j % NMETA;
         HeadMeta& hm = sh.meta[m];
-        wait_or_abort(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
-        CLK_BEGIN(t_a1);
-
-        // ---- a1: top-r of |q| for this unit; key = |q_c| bits above (127 - c)
-        const int n = a.seq_lens[b];
+        // key = |q_c| bits above (127 - c): distinct keys, larger |q| first, then smaller c
+        const int n = n_next;
         const bool valid = n >= 1 && n <= a.S_max;
         const int k_eff = valid ? min(a.k, n) : 0;
         const uint16_t hb[4] = {(uint16_t)(qraw.x & 0xffffu), (uint16_t)(qraw.x >> 16), (uint16_t)(qraw.y & 0xffffu),
                                 (uint16_t)(qraw.y >> 16)};
+        // the next unit's query and length travel while this unit is ranked
+        if (j + 1 < n_mine) {
+            qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)(bh + gridDim.x) * D + lane * 4);
+            n_next = a.seq_lens[(bh + gridDim.x) / a.Hq];
+        }
+        wait_or_abort<200>(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
+        CLK_BEGIN(t_a1);
         float qf[4], l1_all = 0.f;
         uint32_t mine[4];
 #pragma unroll
@@ -150,14 +161,24 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
         }
         __syncwarp();
         if (a.idx_r) for (int c = lane; c < a.r; c += 32) a.idx_r[(size_t)bh * a.r + c] = valid ? hm.i1[c] : -1;
-        // the next unit's query travels while this unit's rows are issued
-        if (j + 1 < n_mine) qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)(bh + gridDim.x) * D + lane * 4);
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.meta_full[m]);
         CLK_ADD(6, t_a1, lane == 0);
+    }
+}
 
-        // ---- issue the unit's ring stages: [chunk c][row batch jb] -> RB rows x CH positions
-        if (k_eff > 0) {
+// ---------------------------------------------------------------------------------- producer
+__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine) {
+    const int lane = threadIdx.x & 31;
+    const int g_heads = a.Hq / a.Hkv;
+    uint32_t g = 0;                                          // ring stages issued so far
+    for (int j = 0; j < n_mine; ++j) {
+        const int m = j % NMETA;
+        const HeadMeta& hm = sh.meta[m];
+        wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        // the unit's ring stages: [chunk c][row batch jb] -> RB rows x CH positions
+        if (hm.k_eff > 0) {
+            const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq, n = hm.n;
             const sparq_half* Kt_head = a.Kt + ((size_t)b * a.Hkv + h / g_heads) * (size_t)D * a.S_max;
             const int n8 = (n + 7) & ~7;
             const int n_chunks = (n8 + CH - 1) / CH;
@@ -167,7 +188,7 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
                     const int s = g % STAGES;
                     const int rows = min(RB, a.r - jb);
                     CLK_BEGIN(t_e);
-                    wait_or_abort(&sh.empty[s], ((g / STAGES) & 1u) ^ 1u, sh, a.status);
+                    wait_or_abort<40>(&sh.empty[s], ((g / STAGES) & 1u) ^ 1u, sh, a.status);
                     CLK_ADD(5, t_e, lane == 0);
                     if (lane == 0) mbar_expect_tx(&sh.full[s], bytes * rows);
                     __syncwarp();
@@ -182,17 +203,19 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
 
 // ---------------------------------------------------------------------------------- stream group
 __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
-                                            int n_mine) {
-    const int gtid = threadIdx.x - 32, lane = gtid & 31;
-    uint32_t g = 0;
+                                            uint32_t* hist1_all, int n_mine) {
+    const int gtid = threadIdx.x - LEAD, lane = gtid & 31;
+    int s = 0;                                               // ring slot and its phase parity
+    uint32_t parity = 0;
     for (int j = 0; j < n_mine; ++j) {
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
+        uint32_t* hist1 = hist1_all + kb * FBINS;
         CLK_BEGIN(t_unit);
-        wait_or_abort(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
         CLK_BEGIN(t_kf);
-        wait_or_abort(&sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
+        wait_or_abort<100>(&sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
         CLK_ADD(2, t_kf, gtid == 0);
         const int n = hm.n, r = a.r;
         if (hm.k_eff > 0) {
@@ -208,31 +231,15 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 for (int e = 0; e < 8; ++e) acc[e] = 0.f;
                 const int t0 = c * CH + gtid * 8;
                 const int nvalid = min(8, n - t0);           // positions of this thread's vector inside the sequence
-                // positions past n in the straddling vector hold whatever the caller's memory holds: mask them
-                uint32_t msk[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
-                for (int jb = 0; jb < r; jb += RB, ++g) {
-                    const int s = g % STAGES;
+                for (int jb = 0; jb < r; jb += RB) {
                     CLK_BEGIN(t_f);
-                    wait_or_abort(&sh.full[s], (g / STAGES) & 1u, sh, a.status);
+                    wait_or_abort<20>(&sh.full[s], parity, sh, a.status);
                     CLK_ADD(3, t_f, gtid == 0);
-                    const uint4* src = reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid;
-                    if (nvalid >= 8) {
-#pragma unroll
-                        for (int u = 0; u < RB; ++u)
-                            if (jb + u < r) row_fma(acc, mx, src[u * (CH / 8)], hm.qh[jb + u]);   // uniform; padded rows were not copied
-                    } else if (nvalid > 0) {
-#pragma unroll
-                        for (int u = 0; u < RB; ++u)
-                            if (jb + u < r) {
-                                uint4 v = src[u * (CH / 8)];
-                                v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
-                                row_fma(acc, mx, v, hm.qh[jb + u]);
-                            }
-                    }
+                    stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid, hm.qh + jb, r - jb,
+                                          nvalid);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sh.empty[s]);   // this warp is done with slot s
+                    if (++s == STAGES) { s = 0; parity ^= 1u; }
                 }
                 uint32_t kk[8];
 #pragma unroll
@@ -241,10 +248,11 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                     *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
                     *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) kmax = max(kmax, kk[e]);
+                    for (int e = 0; e < 8; ++e) { kmax = max(kmax, kk[e]); atomicAdd(&hist1[kk[e] >> FSH], 1u); }
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) if (e < nvalid) { keys[t0 + e] = kk[e]; kmax = max(kmax, kk[e]); }
+                    for (int e = 0; e < 8; ++e)
+                        if (e < nvalid) { keys[t0 + e] = kk[e]; kmax = max(kmax, kk[e]); atomicAdd(&hist1[kk[e] >> FSH], 1u); }
                 }
             }
             uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
@@ -259,9 +267,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 
 // ---------------------------------------------------------------------------------- post groups
 template <class PG>
-__device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, unsigned char* scratch,
-                                          int n_mine, int p) {
-    const int gtid = threadIdx.x - 32 - SNT - p * GNT;
+__device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, uint32_t* hist1_all,
+                                          unsigned char* scratch, int n_mine, int p) {
+    const int gtid = threadIdx.x - LEAD - SNT - p * GNT;
     PostScratch sc;
     carve_post_scratch(sc, scratch, PG::NHW, a.S_cap / 32);
     sc.i2 = sh.i2[p]; sc.red = sh.red[p]; sc.redu = sh.redu[p]; sc.res = sh.res[p]; sc.band = sh.band[p];
@@ -270,7 +278,7 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         CLK_BEGIN(t_w);
-        wait_or_abort(&sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
+        wait_or_abort<100>(&sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
         CLK_ADD(1, t_w, gtid == 0);
         CLK_BEGIN(t_p);
         const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq;
@@ -284,10 +292,15 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             if (gtid < D) out_row[gtid] = a.vbar[kv_head * D + gtid];
             if (gtid == 0 && a.alpha) a.alpha[bh] = 0.f;
         } else {
-            post_phase<PG>(gtid, hm, keys_all + (size_t)kb * a.S_cap, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.k, a.S_max,
-                           a.Kt + kv_head * (size_t)D * a.S_max, a.K + kv_head * (size_t)a.S_max * D,
-                           a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
-                           a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
+            const uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
+            const sparq_half* Kt_head = a.Kt + kv_head * (size_t)D * a.S_max;
+            SelectResult sel;
+            if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, hist1_all + kb * FBINS, a.r, a.S_max,
+                                      Kt_head, sel))
+                sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
+            finish<PG, 4>(gtid, hm, keys, sh.kmax[kb], sel, sc, a.k, a.K + kv_head * (size_t)a.S_max * D,
+                          a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
+                          a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
         }
         PG::sync();                                          // the group is done with the keys, the metadata, i2
         CLK_ADD(0, t_p, gtid == 0);
@@ -299,7 +312,8 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) 
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
     uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);
-    unsigned char* scratch0 = dyn_smem + RING_BYTES + (size_t)NKB * a.S_cap * 4;
+    uint32_t* hist1_all = keys_all + (size_t)NKB * a.S_cap;               // per key buffer: histogram of the keys' top bits
+    unsigned char* scratch0 = reinterpret_cast<unsigned char*>(hist1_all + NKB * FBINS);
     const size_t scratch_bytes = (post_scratch_bytes(GNT / 16, a.S_cap / 32) + 127) & ~(size_t)127;
     __shared__ PipeShared sh;
 
@@ -310,18 +324,20 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) 
         sh.abort_flag = 0;
         mbar_init_fence();
     }
+    for (int i = threadIdx.x; i < NKB * FBINS; i += NT) hist1_all[i] = 0;
     __syncthreads();
     const int n_mine = (a.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units blockIdx.x + j*gridDim.x
     const int warp = threadIdx.x >> 5;
     if (warp == 0) producer_role(a, sh, ring, n_mine);
-    else if (warp <= SNT / 32) stream_role(a, sh, ring, keys_all, n_mine);
-    else if (warp <= SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, scratch0, n_mine, 0);
-    else post_role<PG1>(a, sh, keys_all, scratch0 + scratch_bytes, n_mine, 1);
+    else if (warp == 1) a1_role(a, sh, n_mine);
+    else if (warp < 2 + SNT / 32) stream_role(a, sh, ring, keys_all, hist1_all, n_mine);
+    else if (warp < 2 + SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, hist1_all, scratch0, n_mine, 0);
+    else post_role<PG1>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, n_mine, 1);
 }
 
 size_t pipe_dynamic_smem(int S_cap) {
     const size_t scratch = (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127;
-    return (size_t)RING_BYTES + (size_t)NKB * S_cap * 4 + NPOST * scratch;
+    return (size_t)RING_BYTES + (size_t)NKB * S_cap * 4 + (size_t)NKB * FBINS * 4 + NPOST * scratch;
 }
 
 }  // namespace
