@@ -52,6 +52,7 @@ typedef uint16_t sparq_half;
 
 #define SPARQ_K_MAX 1024
 #define SPARQ_HEAD_DIM 128
+#define SPARQ_STATIC_SCRATCH_BYTES (8u << 20)   /* scratch built into the library for dense_decode_static */
 
 enum {
     SPARQ_OK = 0,
@@ -61,6 +62,8 @@ enum {
     SPARQ_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than *_workspace_bytes()           */
     SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds what the kernels' on-chip score buffer holds   */
     SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
+    SPARQ_ERR_STATIC_SCRATCH = 7,/* the problem needs more scratch than the library's fixed
+                                    SPARQ_STATIC_SCRATCH_BYTES: use the call that takes a workspace */
     SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */
     SPARQ_DEV_CACHE_FULL = 17,   /* device: append with seq_lens[b] == S_max; nothing written    */
     SPARQ_DEV_TIMEOUT = 18       /* device: an asynchronous copy did not land within the bounded wait;
@@ -126,6 +129,34 @@ int dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, 
                  int B, int Hq, int Hkv, int d, int S_max, sparq_half* out,
                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
+
+/*
+ * dense_decode_static -- dense_decode for callers that must not allocate.  (The paper has no
+ * counterpart; this entry point exists for integration only.)
+ *
+ * Who needs it: a decode step that runs inside a host process whose device memory is owned by
+ * someone else -- an inference server that hands its plug-ins fixed buffers and forbids them to call
+ * the allocator, or a latency-critical loop in which an allocation (which may synchronise the whole
+ * device) is not acceptable.  Such a caller cannot create the `workspace` that dense_decode asks
+ * for, so here the scratch for the per-split softmax states is a fixed array of
+ * SPARQ_STATIC_SCRATCH_BYTES (8 MiB) inside the library's own device image.  The call allocates
+ * and frees nothing, on the host API or through any library; q, K, V, seq_lens, out (and status)
+ * are still the caller's buffers, with the same meaning, layout and results as in dense_decode.
+ *
+ * Limits and rules:
+ *   - A problem whose dense_workspace_bytes() exceeds SPARQ_STATIC_SCRATCH_BYTES is refused with
+ *     SPARQ_ERR_STATIC_SCRATCH before anything is launched (use dense_decode with a workspace).
+ *   - The first call on each device looks up the array's device address (a runtime query, not an
+ *     allocation).  Make that first call during set-up, with the device current, and before any
+ *     stream capture is started on that device.
+ *   - Every GPU that loads the library holds the 8 MiB until the process exits, and all calls on a
+ *     device share it.  The array keeps whatever the previous call left; nothing in it needs to be
+ *     zero, because every slot that is read was written earlier in the same call.  Two calls that
+ *     can overlap on the GPU (different streams, or different host threads) race on it: order
+ *     them on one stream or with events.
+ */
+int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                        int B, int Hq, int Hkv, int d, int S_max, sparq_half* out, int32_t* status, void* stream);
 
 /*
  * sparq_step_host -- one whole generation step driven from HOST buffers: copies q_host

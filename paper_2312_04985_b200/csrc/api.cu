@@ -52,6 +52,7 @@ const char* sparq_status_string(int code) {
         case SPARQ_ERR_WORKSPACE: return "SPARQ_ERR_WORKSPACE";
         case SPARQ_ERR_TOO_LONG: return "SPARQ_ERR_TOO_LONG";
         case SPARQ_ERR_CUDA: return "SPARQ_ERR_CUDA";
+        case SPARQ_ERR_STATIC_SCRATCH: return "SPARQ_ERR_STATIC_SCRATCH";
         case SPARQ_DEV_BAD_SEQ_LEN: return "SPARQ_DEV_BAD_SEQ_LEN";
         case SPARQ_DEV_CACHE_FULL: return "SPARQ_DEV_CACHE_FULL";
         case SPARQ_DEV_TIMEOUT: return "SPARQ_DEV_TIMEOUT";
@@ -120,6 +121,17 @@ int dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, 
     if (need && (!workspace || workspace_bytes < need)) return SPARQ_ERR_WORKSPACE;
     return rc(launch_dense_decode(q, K, V, seq_lens, B, Hq, Hkv, S_max, out, (float*)workspace, status,
                                   (cudaStream_t)stream));
+}
+
+int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
+                        int B, int Hq, int Hkv, int d, int S_max, sparq_half* out, int32_t* status, void* stream) {
+    if (!q || !K || !V || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (dense_scratch_bytes(B, Hq, Hkv, S_max) > SPARQ_STATIC_SCRATCH_BYTES) return SPARQ_ERR_STATIC_SCRATCH;
+    float* scratch = nullptr;
+    size_t bytes = 0;
+    if (dense_static_scratch(&scratch, &bytes) != cudaSuccess) return SPARQ_ERR_CUDA;
+    return rc(launch_dense_decode(q, K, V, seq_lens, B, Hq, Hkv, S_max, out, scratch, status, (cudaStream_t)stream));
 }
 
 size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d) {

@@ -3,11 +3,21 @@
 // for all (up to 8 at a time) query heads of its group, so K and V are read once per KV head;
 // half-warp per cache row, 128-bit loads, online softmax in fp32.  With more than one split the
 // per-split softmax states go through a scratch buffer and a small merge kernel.
+#include <mutex>
+
 #include "common.cuh"
 #include "kernels.h"
 
 namespace sparq {
 namespace {
+
+// Scratch of dense_decode_static: lives in the library's device image, so every GPU that loads the
+// library carries these 8 MiB until the process exits, and every call on a device shares them.
+constexpr size_t kStaticScratchBytes = SPARQ_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_dense_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+float* g_dense_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_dense_scratch_mutex;
 
 constexpr int NT = 256;             // threads per CTA
 constexpr int NHW = NT / 16;        // half-warps per CTA (one K/V row each)
@@ -158,6 +168,26 @@ int dense_splits(int B, int Hkv, int S_max) {
 size_t dense_scratch_bytes(int B, int Hq, int Hkv, int S_max) {
     int splits = dense_splits(B, Hkv, S_max);
     return splits == 1 ? 0 : (size_t)B * Hq * splits * (D + 2) * sizeof(float);
+}
+
+// Device address of the static scratch on the current device.  In host code the array's name is only
+// a handle of the symbol, not an address a kernel could use: the address comes from the runtime, once
+// per device, with that device current.
+cudaError_t dense_static_scratch(float** ptr, size_t* bytes) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_dense_scratch_mutex);
+    if (!g_dense_scratch_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_dense_scratch);
+        if (e != cudaSuccess) return e;
+        g_dense_scratch_ptr[dev] = static_cast<float*>(p);
+    }
+    *ptr = g_dense_scratch_ptr[dev];
+    *bytes = kStaticScratchBytes;
+    return cudaSuccess;
 }
 
 cudaError_t launch_dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,

@@ -32,6 +32,8 @@ cudaError_t launch_dense_decode(const sparq_half* q, const sparq_half* K, const 
                                 int B, int Hq, int Hkv, int S_max, sparq_half* out, float* scratch, int32_t* status,
                                 cudaStream_t stream);
 
+cudaError_t dense_static_scratch(float** ptr, size_t* bytes);   // library-owned scratch on the current device
+
 // cache.cu
 cudaError_t launch_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens, sparq_half* Kt,
                                float* vsum, sparq_half* vbar, int B, int Hkv, int S_max, int32_t* status,

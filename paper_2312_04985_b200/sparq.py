@@ -18,13 +18,14 @@ import torch
 from . import build as _build
 
 OK = 0
-ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_BAD_RK, ERR_WORKSPACE, ERR_TOO_LONG, ERR_CUDA = 1, 2, 3, 4, 5, 6
+ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_BAD_RK, ERR_WORKSPACE, ERR_TOO_LONG, ERR_CUDA, ERR_STATIC_SCRATCH = 1, 2, 3, 4, 5, 6, 7
+STATIC_SCRATCH_BYTES = 8 << 20
 DEV_BAD_SEQ_LEN, DEV_CACHE_FULL, DEV_TIMEOUT = 16, 17, 18
 K_MAX = 1024
 HEAD_DIM = 128
 
 EXPORTS = ("sparq_status_string", "sparq_max_seq_len", "sparq_cache_build", "sparq_cache_append", "sparq_decode",
-           "sparq_workspace_bytes", "dense_decode", "dense_workspace_bytes", "sparq_step_host",
+           "sparq_workspace_bytes", "dense_decode", "dense_workspace_bytes", "dense_decode_static", "sparq_step_host",
            "sparq_step_host_staging_bytes")
 
 
@@ -63,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.dense_decode.argtypes = [vp] * 4 + [i] * 5 + [vp, vp, sz, vp, vp]
         L.dense_workspace_bytes.restype = sz
         L.dense_workspace_bytes.argtypes = [i] * 5
+        L.dense_decode_static.restype = i
+        L.dense_decode_static.argtypes = [vp] * 4 + [i] * 5 + [vp, vp, vp]
         L.sparq_step_host.restype = i
         L.sparq_step_host.argtypes = [vp] * 9 + [i] * 7 + [vp, vp, sz, vp, vp]
         L.sparq_step_host_staging_bytes.restype = sz
@@ -160,6 +163,21 @@ def dense_decode(q, K, V, seq_lens, out, workspace=None, status=None):
                                 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                 _dev(status, torch.int32, "status"), _stream(q))
     _check("dense_decode", rc)
+    return out
+
+
+def dense_decode_static(q, K, V, seq_lens, out, status=None):
+    """dense_decode on the library's built-in scratch: no workspace argument, nothing allocated by the
+    call.  Raises SparqError(ERR_STATIC_SCRATCH) when the problem needs more than STATIC_SCRATCH_BYTES.
+    Calls on one device share that scratch: keep them ordered on one stream."""
+    B, Hq, d = q.shape
+    Hkv, S_max = K.shape[1], K.shape[2]
+    with torch.cuda.device(q.device):
+        rc = lib().dense_decode_static(_dev(q, torch.float16, "q"), _dev(K, torch.float16, "K"),
+                                       _dev(V, torch.float16, "V"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                       B, Hq, Hkv, d, S_max, _dev(out, torch.float16, "out"),
+                                       _dev(status, torch.int32, "status"), _stream(q))
+    _check("dense_decode_static", rc)
     return out
 
 
