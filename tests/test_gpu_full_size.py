@@ -1,0 +1,114 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times: every
+(batch, head) unit is checked against properties that hold at any size, and a seeded sample of
+units element by element against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import c_oracle
+from paper_2312_04985_b200 import sparq, synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+class FullCache:
+    """Device-resident workload of a Case generated on the GPU (no host copy of the whole cache)."""
+
+    def __init__(self, case):
+        dev = case.K.device
+        self.c = case
+        self.K, self.V = case.K, case.V
+        B, Hkv, S_max, d = self.K.shape
+        self.seq = case.seq_lens.clone()
+        self.Kt = torch.zeros(B, Hkv, d, S_max, dtype=torch.float16, device=dev)
+        self.vsum = torch.zeros(B, Hkv, d, dtype=torch.float32, device=dev)
+        self.vbar = torch.zeros(B, Hkv, d, dtype=torch.float16, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        sparq.sparq_cache_build(self.K, self.V, self.seq, self.Kt, self.vsum, self.vbar, self.status)
+
+    def step(self, i):
+        c = self.c
+        sparq.sparq_cache_append(c.k_steps[i], c.v_steps[i], self.K, self.Kt, self.V, self.vsum, self.vbar, self.seq,
+                                 self.status)
+        out = torch.empty(c.B, c.Hq, c.d, dtype=torch.float16, device=self.K.device)
+        i1 = torch.empty(c.B, c.Hq, c.r, dtype=torch.int32, device=self.K.device)
+        i2 = torch.empty(c.B, c.Hq, c.k, dtype=torch.int32, device=self.K.device)
+        al = torch.empty(c.B, c.Hq, dtype=torch.float32, device=self.K.device)
+        sparq.sparq_decode(c.q_steps[i], self.K, self.Kt, self.V, self.vbar, self.seq, c.r, c.k, out, idx_r=i1, idx_k=i2,
+                           alpha=al, status=self.status)
+        torch.cuda.synchronize()
+        return out, i1, i2, al
+
+
+def check_all_units_properties(fc, out, i1, i2, al):
+    c = fc.c
+    n = fc.seq.view(-1, 1, 1).to(torch.int64)
+    assert torch.isfinite(out.float()).all()
+    assert ((al >= 0) & (al <= 1 + 1e-5)).all()                                  # alpha is a probability mass
+    assert (i1[..., 1:] > i1[..., :-1]).all() and (i1 >= 0).all() and (i1 < c.d).all()      # sets, ascending
+    assert (i2[..., 1:] > i2[..., :-1]).all() and (i2 >= 0).all() and (i2 < n).all()        # k <= n in these workloads
+
+
+def check_top_r_property(q, i1, r):
+    a = q.float().abs()
+    sel = torch.zeros_like(a, dtype=torch.bool).scatter_(2, i1.to(torch.int64), True)
+    weakest_in = torch.where(sel, a, torch.full_like(a, float("inf"))).min(dim=2).values
+    strongest_out = torch.where(sel, torch.full_like(a, -1.0), a).max(dim=2).values
+    assert (weakest_in >= strongest_out).all()
+
+
+def check_sampled_units(fc, q, out, i1, i2, al, n_sample, what, seed=0):
+    c = fc.c
+    g = torch.Generator().manual_seed(seed)
+    flat = torch.randperm(c.B * c.Hq, generator=g)[:n_sample]
+    bs, hs = (flat // c.Hq).tolist(), (flat % c.Hq).tolist()
+    grp = c.Hq // c.Hkv
+    Ku = torch.stack([fc.K[b, h // grp] for b, h in zip(bs, hs)]).unsqueeze(1).cpu().numpy()
+    Vu = torch.stack([fc.V[b, h // grp] for b, h in zip(bs, hs)]).unsqueeze(1).cpu().numpy()
+    qu = torch.stack([q[b, h] for b, h in zip(bs, hs)]).unsqueeze(1).cpu().numpy()
+    seq = fc.seq.cpu()[torch.tensor(bs)].numpy().astype(np.int32)
+    ora = c_oracle.sparq_decode(qu, Ku, Vu, seq, c.r, c.k)
+    gpu = dict(out=torch.stack([out[b, h] for b, h in zip(bs, hs)]).cpu().numpy().astype(np.float64),
+               i1=torch.stack([i1[b, h] for b, h in zip(bs, hs)]).cpu().numpy(),
+               i2=torch.stack([i2[b, h] for b, h in zip(bs, hs)]).cpu().numpy(),
+               alpha=torch.stack([al[b, h] for b, h in zip(bs, hs)]).cpu().numpy().astype(np.float64))
+    waived = H.compare_units(gpu, ora, qu[:, 0], lambda u: Ku[u, 0], lambda u: Vu[u, 0], seq, c.r, c.k, what)
+    assert waived <= max(1, n_sample // 50)
+
+
+@pytest.mark.parametrize("name,n_sample", [("c2", 64), ("c3", 48)])
+def test_full_size_single_step(name, n_sample):
+    c = synth.make_case(name, device="cuda")
+    fc = FullCache(c)
+    out, i1, i2, al = fc.step(0)
+    assert int(fc.status.item()) == 0
+    assert fc.seq.tolist() == [synth.SPECS[name]["S"]] * c.B
+    check_all_units_properties(fc, out, i1, i2, al)
+    check_top_r_property(c.q_steps[0], i1, c.r)
+    check_sampled_units(fc, c.q_steps[0], out, i1, i2, al, n_sample, name)
+    # the appended row landed in all three cache tensors
+    S = c.S_max
+    assert torch.equal(fc.Kt[:, :, :, S - 1], c.k_steps[0]) and torch.equal(fc.K[:, :, S - 1], c.k_steps[0])
+    assert torch.equal(fc.V[:, :, S - 1], c.v_steps[0])
+
+
+def test_full_size_c4_32_append_decode_steps():
+    c = synth.make_case("c4", device="cuda")
+    assert (c.B, c.Hq, c.Hkv, c.S_max, c.r, c.k, c.n_steps) == (16, 32, 8, 32800, 64, 256, 32)
+    fc = FullCache(c)
+    seq0 = fc.seq.clone()
+    for i in range(c.n_steps):
+        out, i1, i2, al = fc.step(i)
+        check_all_units_properties(fc, out, i1, i2, al)
+        if i in (0, 15, 31):
+            check_top_r_property(c.q_steps[i], i1, c.r)
+            check_sampled_units(fc, c.q_steps[i], out, i1, i2, al, 16, "c4 step %d" % i, seed=i)
+    assert int(fc.status.item()) == 0
+    assert torch.equal(fc.seq, seq0 + c.n_steps)
+    # after 32 appends: Kt is the transpose of K on the valid rows and v_bar their mean (sampled heads)
+    for b, h in ((0, 0), (7, 3), (15, 7)):
+        n = int(fc.seq[b])
+        assert torch.equal(fc.Kt[b, h, :, :n], fc.K[b, h, :n].t())
+        mean = fc.V[b, h, :n].double().mean(0)
+        assert (fc.vbar[b, h].double() - mean).abs().max() < 2e-4

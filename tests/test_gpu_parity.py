@@ -60,7 +60,7 @@ def test_shrunk_batch_all_heads(name, kw):
 
 def test_more_units_than_sms_all_heads():
     """More (batch, head) units than SMs, so the persistent kernel's CTAs each walk several units
-    (ring, key-buffer and metadata slots wrap around) with ragged lengths and an invalid sequence."""
+    (ring, key-buffer and metadata slots wrap around) with ragged lengths."""
     c = synth.make_case("c2", device="cuda", B=21, S=1024, ragged=(700, 1023))       # 672 units
     c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
                                                                                   c.v_steps, c.seq_lens))
