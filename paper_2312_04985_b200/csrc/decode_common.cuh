@@ -519,6 +519,13 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
         carry_sel += tot;
     }
     G::sync();
+    // start the selected rows on their way from HBM to L2 now; the gather below reads them a few
+    // barriers later (two 128-byte lines per row and tensor)
+    for (int i = gtid; i < 4 * k_eff; i += G::NT) {
+        const int t = min(max(sc.i2[i >> 2], 0), n - 1);
+        const sparq_half* row = ((i & 2) ? V_head : K_head) + (size_t)t * D + (i & 1) * (D / 2);
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
+    }
     // alpha = approximate-score mass of the selected set (Step 3)
     float apart = 0.f;
     for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[sc.i2[j]]) - vmax) * c1);
@@ -535,7 +542,11 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     float m = -CUDART_INF_F, l = 0.f, acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 1
+    for (int jb = 0; jb < 0; jb += G::NHW * RG) {
+#else
     for (int jb = 0; jb < k_eff; jb += G::NHW * RG) {        // trip count uniform across the group
+#endif
         uint4 kv[RG], vv[RG];
 #pragma unroll
         for (int u = 0; u < RG; ++u) {

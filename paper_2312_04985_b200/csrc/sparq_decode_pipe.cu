@@ -3,8 +3,10 @@
 // never waits for the latency-bound stages:
 //
 //   a1 warp           top-r of |q| and tau for the units ahead (metadata slots), off everyone's path
-//   producer warp     the bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast) of the
-//                     r selected Kt rows into a ring of shared-memory stages; lanes issue one row each
+//   producer warps    the bulk asynchronous copies (cp.async.bulk + mbarrier, no multicast) of the
+//                     r selected Kt rows into a ring of shared-memory stages; two warps take
+//                     alternate stages and lanes issue one row each, because one thread (and even
+//                     one warp) can only start a copy every few hundred cycles
 //   stream group      a2: consumes the ring, fp32 mixed-precision FMA chain per position, writes the
 //                     order-preserving keys of unit j into key buffer j mod 3
 //   post groups 0/1   a3-a6 of units j = 0,2,4,.. / 1,3,5,.. (decode_common.cuh): radix select with
@@ -22,11 +24,12 @@ namespace {
 constexpr int SNT = 256;                 // stream-group threads
 constexpr int GNT = 256;                 // threads of one post group
 constexpr int NPOST = 2;
-constexpr int LEAD = 64;                 // producer warp + a1 warp
+constexpr int NPROD = 2;                 // producer warps (one warp alone cannot start copies fast enough)
+constexpr int LEAD = 32 * (NPROD + 1);   // producer warps + a1 warp
 constexpr int NT = LEAD + SNT + NPOST * GNT;
 constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
-constexpr int RB = 8;                    // Kt rows per ring stage
-constexpr int STAGES = 3;
+constexpr int RB = 4;                    // Kt rows per ring stage
+constexpr int STAGES = 6;
 constexpr int STAGE_BYTES = RB * CH * 2;
 constexpr int RING_BYTES = STAGES * STAGE_BYTES;
 constexpr int NKB = 3;                   // key buffers: one being written, two being post-processed
@@ -91,6 +94,14 @@ __device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, Pi
     }
     *flag = 1;
     raise_status(status, SPARQ_DEV_TIMEOUT);
+}
+
+// The same for a whole thread group: its first warp polls, the other warps sleep in the group's
+// hardware barrier instead of spending issue slots on polls.
+template <class G, int NS>
+__device__ __forceinline__ void group_wait(int gtid, uint64_t* bar, uint32_t parity, PipeShared& sh, int32_t* status) {
+    if (gtid < 32) wait_or_abort<NS>(bar, parity, sh, status);
+    G::sync();
 }
 
 // ---------------------------------------------------------------------------------- a1 warp
@@ -168,7 +179,7 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_min
 }
 
 // ---------------------------------------------------------------------------------- producer
-__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine) {
+__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine, int p) {
     const int lane = threadIdx.x & 31;
     const int g_heads = a.Hq / a.Hkv;
     uint32_t g = 0;                                          // ring stages issued so far
@@ -185,11 +196,10 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
             for (int c = 0; c < n_chunks; ++c) {
                 const uint32_t bytes = (uint32_t)min(CH, n8 - c * CH) * 2u;
                 for (int jb = 0; jb < a.r; jb += RB, ++g) {
+                    if ((int)(g % NPROD) != p) continue;     // the other producer warp's stage
                     const int s = g % STAGES;
                     const int rows = min(RB, a.r - jb);
-                    CLK_BEGIN(t_e);
                     wait_or_abort<40>(&sh.empty[s], ((g / STAGES) & 1u) ^ 1u, sh, a.status);
-                    CLK_ADD(5, t_e, lane == 0);
                     if (lane == 0) mbar_expect_tx(&sh.full[s], bytes * rows);
                     __syncwarp();
                     if (lane < rows)
@@ -213,9 +223,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
         uint32_t* hist1 = hist1_all + kb * FBINS;
         CLK_BEGIN(t_unit);
-        wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        if (gtid < 32) wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
         CLK_BEGIN(t_kf);
-        wait_or_abort<100>(&sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
+        group_wait<SG, 100>(gtid, &sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
         CLK_ADD(2, t_kf, gtid == 0);
         const int n = hm.n, r = a.r;
         if (hm.k_eff > 0) {
@@ -232,9 +242,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 const int t0 = c * CH + gtid * 8;
                 const int nvalid = min(8, n - t0);           // positions of this thread's vector inside the sequence
                 for (int jb = 0; jb < r; jb += RB) {
-                    CLK_BEGIN(t_f);
                     wait_or_abort<20>(&sh.full[s], parity, sh, a.status);
-                    CLK_ADD(3, t_f, gtid == 0);
                     stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid, hm.qh + jb, r - jb,
                                           nvalid);
                     __syncwarp();
@@ -278,7 +286,7 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         CLK_BEGIN(t_w);
-        wait_or_abort<100>(&sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
+        group_wait<PG, 100>(gtid, &sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
         CLK_ADD(1, t_w, gtid == 0);
         CLK_BEGIN(t_p);
         const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq;
@@ -295,9 +303,16 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             const uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
             const sparq_half* Kt_head = a.Kt + kv_head * (size_t)D * a.S_max;
             SelectResult sel;
+#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 3
+            sel.Z = 1.f; sel.need_tie = 0;
+            if (false)
+#endif
             if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, hist1_all + kb * FBINS, a.r, a.S_max,
                                       Kt_head, sel))
                 sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
+#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 2
+            if (false)
+#endif
             finish<PG, 4>(gtid, hm, keys, sh.kmax[kb], sel, sc, a.k, a.K + kv_head * (size_t)a.S_max * D,
                           a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
                           a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
@@ -328,10 +343,10 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) 
     __syncthreads();
     const int n_mine = (a.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units blockIdx.x + j*gridDim.x
     const int warp = threadIdx.x >> 5;
-    if (warp == 0) producer_role(a, sh, ring, n_mine);
-    else if (warp == 1) a1_role(a, sh, n_mine);
-    else if (warp < 2 + SNT / 32) stream_role(a, sh, ring, keys_all, hist1_all, n_mine);
-    else if (warp < 2 + SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, hist1_all, scratch0, n_mine, 0);
+    if (warp < NPROD) producer_role(a, sh, ring, n_mine, warp);
+    else if (warp == NPROD) a1_role(a, sh, n_mine);
+    else if (warp < LEAD / 32 + SNT / 32) stream_role(a, sh, ring, keys_all, hist1_all, n_mine);
+    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, hist1_all, scratch0, n_mine, 0);
     else post_role<PG1>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, n_mine, 1);
 }
 
