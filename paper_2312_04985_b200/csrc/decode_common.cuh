@@ -7,6 +7,15 @@
 
 namespace sparq {
 
+#ifdef SPARQ_PHASE_CLOCKS
+__device__ unsigned long long g_post_clocks[16];
+#define POST_CLK_INIT() long long pc_prev_ = clock64()
+#define POST_CLK(i) do { if (gtid == 0) { long long pc_now_ = clock64(); atomicAdd(&g_post_clocks[i], (unsigned long long)(pc_now_ - pc_prev_)); pc_prev_ = pc_now_; } } while (0)
+#else
+#define POST_CLK_INIT()
+#define POST_CLK(i)
+#endif
+
 constexpr int HIST_BINS = 2048;
 constexpr int CAND_MAX = 256;            // threshold-band positions the quick fp64 re-decision handles
 constexpr int WAIT_LIMIT = 1 << 22;      // polls before an asynchronous copy is declared lost
@@ -25,6 +34,7 @@ struct Group {
 // What the later stages need to know about one (batch, query head) unit; filled by stage a1.
 struct alignas(16) HeadMeta {
     float qf[D];                  // q as fp32
+    uint16_t q16[D];              // q as stored (fp16 bits)
     int32_t i1[D];                // selected components, ascending
     uint32_t rkey[D];             // a1 scratch: ranking keys
     uint16_t qh[D + 8];           // selected components' fp16 bits in i1 order, zero padded
@@ -372,8 +382,8 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // keys builds the bitmap of everything above the threshold bin, the softmax denominator and the list
 // of the bin's own keys; the threshold is then resolved inside that short list, and the 2B band
 // around it re-decided in fp64 as in select_generic.  Clears hist1 for its next user.
-// Returns false (for every thread of the group alike) when the short-cut does not apply -- the bin
-// holds more keys than the list, or the band reaches outside the bin or holds too many keys -- and
+// Returns false (for every thread of the group alike) when the short-cut does not apply -- a warp
+// meets more of the bin's keys than its list segment holds, or the band reaches outside the bin or holds too many keys -- and
 // the caller runs select_generic instead.
 template <class G>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
@@ -385,32 +395,58 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const float vmax = unkey32(kmax);
     const float c1 = hm.inv_tau * LOG2E;
 
-    if (gtid < 4) sc.band[gtid] = 0;     // [0] band keys below the edge, [1] at/above it, [2] band list, [3] bin list
+    POST_CLK_INIT();
+    if (gtid < 4) sc.band[gtid] = 0;     // [0] band keys below the edge, [1] at/above it, [2] band list length
     find_bin<G, FBINS>(hist1, (uint32_t)k_eff, sc.redu, sc.res, gtid);
+    POST_CLK(0);
     const uint32_t b1 = sc.res[0], above = sc.res[1];
     for (int i = gtid; i < FBINS / 4; i += G::NT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
-    uint32_t* list_key = sc.hist;
-    int32_t* list_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX);
+    // the bin's own keys: every warp appends to its own segment of the list (no atomics), in the
+    // order it meets them
+    constexpr int SEG = LIST_MAX / G::NW;                    // (key, position) pairs per warp
+    uint32_t* seg_key = sc.hist + warp * SEG;
+    int32_t* seg_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX) + warp * SEG;
+    const unsigned lt = (1u << lane) - 1;
 
     const int nwords = (n + 31) >> 5;
     float zpart = 0.f;
-    for (int wi = warp; wi < nwords; wi += G::NW) {
-        const int t = (wi << 5) + lane;
-        const bool valid = t < n;
-        const uint32_t u = valid ? keys[t] : 0u;
-        zpart += valid ? ex2((unkey32(u) - vmax) * c1) : 0.f;
-        const uint32_t dig = u >> FSH;
-        const unsigned g = __ballot_sync(FULL, valid && dig > b1);
-        if (lane == 0) sc.bm_sel[wi] = g;
-        if (valid && dig == b1) {
-            const uint32_t slot = atomicAdd(&sc.band[3], 1u);
-            if (slot < LIST_MAX) { list_key[slot] = u; list_pos[slot] = t; }
+    uint32_t wcount = 0;                                     // this warp's list length (warp-uniform)
+    for (int w0 = warp; w0 < nwords; w0 += 4 * G::NW) {      // four words in flight per warp
+        uint32_t u[4];
+        bool valid[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int t = ((w0 + x * G::NW) << 5) + lane;
+            valid[x] = t < n;                                // also false for words past the end
+            u[x] = valid[x] ? keys[t] : 0u;
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int wi = w0 + x * G::NW;
+            if (wi < nwords) {                               // warp-uniform
+                zpart += valid[x] ? ex2((unkey32(u[x]) - vmax) * c1) : 0.f;
+                const uint32_t dig = u[x] >> FSH;
+                const unsigned g = __ballot_sync(FULL, valid[x] && dig > b1);
+                const unsigned inb = __ballot_sync(FULL, valid[x] && dig == b1);
+                if (lane == 0) sc.bm_sel[wi] = g;
+                if (inb) {
+                    const uint32_t slot = wcount + __popc(inb & lt);
+                    if ((inb >> lane & 1u) && slot < SEG) { seg_key[slot] = u[x]; seg_pos[slot] = (wi << 5) + lane; }
+                    wcount += __popc(inb);
+                }
+            }
         }
     }
-    out.Z = group_sum<G>(zpart, sc.red, gtid);               // barriers also publish the bitmap and the list
+    if (lane == 0) sc.redu[G::NW + warp] = wcount;           // second half of redu: free during group_sum
+    out.Z = group_sum<G>(zpart, sc.red, gtid);               // barriers also publish the bitmap and the lists
     out.need_tie = 0;
-    const uint32_t m = sc.band[3];
-    if (m > LIST_MAX) return false;
+    POST_CLK(1);
+    uint32_t m = 0;
+    bool fits = true;
+#pragma unroll
+    for (int w = 0; w < G::NW; ++w) { const uint32_t c = sc.redu[G::NW + w]; m += c; fits = fits && c <= SEG; }
+    if (!fits) return false;
+    const uint32_t my_n = min(wcount, (uint32_t)SEG);
 
     // the threshold among the bin's m keys: `need` of them are wanted; remaining 22 bits as 8 + 8 + 6
     uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH, mask = ~0u << FSH, ceq = m;
@@ -422,8 +458,8 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         shift -= bits;
         if (gtid < 256) h256[gtid] = 0;
         G::sync();
-        for (uint32_t i = gtid; i < m; i += G::NT) {
-            const uint32_t u = list_key[i];
+        for (uint32_t i = lane; i < my_n; i += 32) {
+            const uint32_t u = seg_key[i];
             if ((u & mask) == prefix) atomicAdd(&h256[(u >> shift) & ((1u << bits) - 1)], 1u);
         }
         G::sync();
@@ -449,6 +485,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         need -= sc.res[1];
         ceq = sc.res[2];
     }
+    POST_CLK(2);
     const uint32_t edge = prefix;                            // unprocessed low bits are zero
     const uint32_t over = ceq - need;
     const float twoB = two_b(r, hm.l1_sel, kabs);
@@ -456,9 +493,9 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
     if ((lo_key >> FSH) != b1 || (hi_key >> FSH) != b1) return false;   // keys outside the list may be in the band
 
-    for (uint32_t i = gtid; i < m; i += G::NT) {
-        const uint32_t u = list_key[i];
-        const int t = list_pos[i];
+    for (uint32_t i = lane; i < my_n; i += 32) {
+        const uint32_t u = seg_key[i];
+        const int t = seg_pos[i];
         if (u >= edge) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
         if (u >= lo_key && u <= hi_key) {
             atomicAdd(&sc.band[u >= edge ? 1 : 0], 1u);
@@ -472,6 +509,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         if (n_cand > CAND_MAX) return false;
         redecide_band<G>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
     }
+    POST_CLK(3);
     return true;
 }
 
@@ -492,6 +530,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     const float c1 = hm.inv_tau * LOG2E;
     const float Z = sel.Z;
     const uint32_t need_tie = sel.need_tie;
+    POST_CLK_INIT();
 
     // ascending list of selected positions from the bitmap(s)
     uint32_t carry_tie = 0, carry_sel = 0;
@@ -530,13 +569,13 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     float apart = 0.f;
     for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[sc.i2[j]]) - vmax) * c1);
     const float alpha = group_sum<G>(apart, sc.red, gtid) / Z;
+    POST_CLK(4);
 
     // -------------------------------------------------------------- a5: gather k rows of K and V
     const int hw = gtid >> 4, l16 = gtid & 15;
     const float qscale = rsqrtf((float)D) * LOG2E;
-    float qs[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) qs[e] = hm.qf[l16 * 8 + e] * qscale;
+    const uint4 q8 = *reinterpret_cast<const uint4*>(hm.q16 + l16 * 8);   // this lane's 8 query components, fp16
+    const uint32_t qw[4] = {q8.x, q8.y, q8.z, q8.w};
     const uint4* Kh = reinterpret_cast<const uint4*>(K_head);
     const uint4* Vh = reinterpret_cast<const uint4*>(V_head);
     float m = -CUDART_INF_F, l = 0.f, acc[8];
@@ -558,14 +597,14 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
         float z[RG], bmax = -CUDART_INF_F;
 #pragma unroll
         for (int u = 0; u < RG; ++u) {
-            const __half2* kh = reinterpret_cast<const __half2*>(&kv[u]);
-            float zz = 0.f;
+            const uint32_t kw[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+            float zz = 0.f, zz2 = 0.f;                       // exact fp16 products, two fp32 chains
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float2 f = __half22float2(kh[e]);
-                zz = fmaf(f.x, qs[2 * e], zz);
-                zz = fmaf(f.y, qs[2 * e + 1], zz);
+                fma_h(zz, (uint16_t)(kw[e] & 0xffffu), (uint16_t)(qw[e] & 0xffffu));
+                fma_h(zz2, (uint16_t)(kw[e] >> 16), (uint16_t)(qw[e] >> 16));
             }
+            zz = (zz + zz2) * qscale;
 #pragma unroll
             for (int o = 8; o > 0; o >>= 1) zz += __shfl_xor_sync(FULL, zz, o);
             z[u] = (jb + u * G::NHW + hw < k_eff) ? zz : -CUDART_INF_F;   // uniform within the half-warp
@@ -592,6 +631,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
             m = mn;
         }
     }
+    POST_CLK(5);
     // merge the half-warps' partial softmax states
     float* mg = sc.merge + hw * (D + 2);
 #pragma unroll
@@ -616,6 +656,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     }
     if (gtid == 0 && alpha_out) *alpha_out = alpha;
     if (idx_k_row) for (int j = gtid; j < k; j += G::NT) idx_k_row[j] = (j < k_eff) ? sc.i2[j] : -1;
+    POST_CLK(6);
 }
 
 }  // namespace sparq

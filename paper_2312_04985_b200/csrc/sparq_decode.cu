@@ -104,6 +104,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         aq = fabsf(qf);
         mine = ((uint32_t)(hb & 0x7fffu) << 7) | (uint32_t)(D - 1 - tid);
         hm.qf[tid] = qf;
+        hm.q16[tid] = hb;
         hm.rkey[tid] = mine;
     }
     __syncthreads();

@@ -139,6 +139,7 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_min
             l1_all += fabsf(qf[e]);
             mine[e] = ((uint32_t)(hb[e] & 0x7fffu) << 7) | (uint32_t)(D - 1 - c);
             hm.qf[c] = qf[e];
+            hm.q16[c] = hb[e];
             hm.rkey[c] = mine[e];
         }
         __syncwarp();
@@ -362,6 +363,12 @@ extern "C" int sparq_debug_pipe_clocks(unsigned long long* out16, int reset) {
     cudaDeviceSynchronize();
     if (out16 && cudaMemcpyFromSymbol(out16, g_pipe_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
     if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_pipe_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+extern "C" int sparq_debug_post_clocks(unsigned long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    if (out16 && cudaMemcpyFromSymbol(out16, g_post_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_post_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
     return 0;
 }
 #endif
