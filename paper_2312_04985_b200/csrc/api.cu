@@ -27,13 +27,16 @@ int device_sm_count() {
     return v;
 }
 
-// SPARQ_DECODE_PLAN=simple|pipe forces one of the two sparq_decode kernels (tests and tuning);
-// unset or anything else: the persistent pipelined kernel whenever its buffers fit.
+// SPARQ_DECODE_PLAN=simple|pipe|split forces one of the sparq_decode plans (tests and tuning).
+// Unset or anything else: the split-S plan when there are fewer units than SMs and the caller
+// passed its workspace, else the persistent pipelined kernel whenever its buffers fit, else one
+// CTA per unit.
 int forced_plan() {
     const char* e = getenv("SPARQ_DECODE_PLAN");
     if (!e) return 0;
     if (!strcmp(e, "simple")) return 1;
     if (!strcmp(e, "pipe")) return 2;
+    if (!strcmp(e, "split")) return 3;
     return 0;
 }
 
@@ -85,19 +88,29 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
                                   (cudaStream_t)stream));
 }
 
-size_t sparq_workspace_bytes(int, int, int, int, int, int, int) { return 0; }
+size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
+    (void)r; (void)k;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
+    const int splits = split_count(B * Hq, S_max, device_sm_count());
+    return splits ? split_scratch_bytes(B * Hq, S_max, splits) : 0;
+}
 
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                  const sparq_half* vbar, const int32_t* seq_lens,
                  int B, int Hq, int Hkv, int d, int S_max, int r, int k,
                  sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
-    (void)workspace; (void)workspace_bytes;
     if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
     if (S_max > sparq_max_seq_len()) return SPARQ_ERR_TOO_LONG;
     const int plan = forced_plan();
+    const int splits = split_count(B * Hq, S_max, device_sm_count());
+    const bool ws_ok = splits && workspace && workspace_bytes >= split_scratch_bytes(B * Hq, S_max, splits);
+    if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
+    if (ws_ok && (plan == 0 || plan == 3))
+        return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
+                                            alpha, status, splits, workspace, (cudaStream_t)stream));
     const bool fits = pipe_fits(S_max, device_smem_optin());
     if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
     if (fits && plan != 1)

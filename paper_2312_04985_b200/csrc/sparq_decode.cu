@@ -48,6 +48,54 @@ __device__ unsigned long long g_phase_clocks[16];
 #define PHASE_MARK(i)
 #endif
 
+// Stage a1 by a whole CTA (G::NT >= 128 threads): the r largest |q_j| by rank counting.
+// key = |q_j| bit pattern above (127 - j): distinct keys, larger |q| first, then smaller j.
+// Fills hm.qf, q16, i1 (ascending), qh (zero padded to a multiple of RB_), inv_tau, l1_sel.
+// red: 2*NW floats, cnt: 4 words.  Ends with a barrier.
+template <class G, int RB_>
+__device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restrict__ q_row, int r, HeadMeta& hm, float* red,
+                                            uint32_t* cnt) {
+    const int lane = tid & 31, warp = tid >> 5;
+    uint16_t hb = 0;
+    float qf = 0.f, aq = 0.f;
+    uint32_t mine = 0;
+    if (tid < D) {
+        hb = q_row[tid];
+        qf = __half2float(__ushort_as_half(hb));
+        aq = fabsf(qf);
+        mine = ((uint32_t)(hb & 0x7fffu) << 7) | (uint32_t)(D - 1 - tid);
+        hm.qf[tid] = qf;
+        hm.q16[tid] = hb;
+        hm.rkey[tid] = mine;
+    }
+    G::sync();
+    bool sel = false;
+    if (tid < D) {
+        int rank = 0;
+        const uint4* rk4 = reinterpret_cast<const uint4*>(hm.rkey);
+#pragma unroll 8
+        for (int j = 0; j < D / 4; ++j) {
+            uint4 o = rk4[j];
+            rank += (o.x > mine) + (o.y > mine) + (o.z > mine) + (o.w > mine);
+        }
+        sel = rank < r;
+    }
+    const unsigned bal = __ballot_sync(FULL, sel);
+    if (lane == 0 && warp < 4) cnt[warp] = __popc(bal);      // warps 0..3 hold the D components
+    float l1_all = aq, l1_sel = sel ? aq : 0.f;
+    group_sum2<G>(l1_all, l1_sel, red, tid);                 // its barriers also publish cnt
+    if (sel) {
+        int slot = __popc(bal & ((1u << lane) - 1));
+        for (int w = 0; w < warp; ++w) slot += cnt[w];
+        hm.i1[slot] = tid;                                   // ascending by construction
+        hm.qh[slot] = hb;
+    }
+    const int r_pad = (r + RB_ - 1) / RB_ * RB_;
+    if (tid >= r && tid < r_pad) hm.qh[tid] = 0;
+    if (tid == 0) { hm.inv_tau = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f; hm.l1_sel = l1_sel; }
+    G::sync();
+}
+
 struct DecodeShared {
     HeadMeta hm;
     int32_t i2[SPARQ_K_MAX];
@@ -58,13 +106,18 @@ struct DecodeShared {
     uint32_t band[4];
 };
 
+// FROM_SCRATCH = false: the whole step.  FROM_SCRATCH = true: the second kernel of the split-S plan;
+// the keys of this unit were written to ws_keys by sparq_split_scores_kernel (with per-split maxima
+// in ws_part), so a2 is replaced by a copy of the keys into shared memory.
+template <bool FROM_SCRATCH>
 __global__ void __launch_bounds__(NT, 3)
 sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                     const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
                     const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
                     int Hq, int Hkv, int S_max, int r, int k,
                     sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
-                    float* __restrict__ alpha_out, int32_t* status) {
+                    float* __restrict__ alpha_out, int32_t* status,
+                    const uint32_t* __restrict__ ws_keys, const uint32_t* __restrict__ ws_part, int splits) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;                                       // a2: STAGES x [RB rows x CH positions] fp16
     uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);  // [n] approximate-score keys
@@ -93,46 +146,8 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = 1;
     }
 
-    // ------------------------------------------------------------------ a1: top-r of |q|
-    // key = |q_j| bit pattern above (127 - j): distinct keys, larger |q| first, then smaller j.
-    uint16_t hb = 0;
-    float qf = 0.f, aq = 0.f;
-    uint32_t mine = 0;
-    if (tid < D) {
-        hb = q[(size_t)bh * D + tid];
-        qf = __half2float(__ushort_as_half(hb));
-        aq = fabsf(qf);
-        mine = ((uint32_t)(hb & 0x7fffu) << 7) | (uint32_t)(D - 1 - tid);
-        hm.qf[tid] = qf;
-        hm.q16[tid] = hb;
-        hm.rkey[tid] = mine;
-    }
-    __syncthreads();
-    bool sel = false;
-    if (tid < D) {
-        int rank = 0;
-        const uint4* rk4 = reinterpret_cast<const uint4*>(hm.rkey);
-#pragma unroll 8
-        for (int j = 0; j < D / 4; ++j) {
-            uint4 o = rk4[j];
-            rank += (o.x > mine) + (o.y > mine) + (o.z > mine) + (o.w > mine);
-        }
-        sel = rank < r;
-    }
-    const unsigned bal = __ballot_sync(FULL, sel);
-    if (lane == 0 && warp < 4) sh.res[warp] = __popc(bal);   // warps 0..3 hold the D components
-    float l1_all = aq, l1_sel = sel ? aq : 0.f;
-    group_sum2<CTA>(l1_all, l1_sel, sh.red, tid);            // its barriers also publish res
-    if (sel) {
-        int slot = __popc(bal & ((1u << lane) - 1));
-        for (int w = 0; w < warp; ++w) slot += sh.res[w];
-        hm.i1[slot] = tid;                                   // ascending by construction
-        hm.qh[slot] = hb;
-    }
+    top_r_block<CTA, RB>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.res);        // a1
     const int r_pad = (r + RB - 1) / RB * RB;
-    if (tid >= r && tid < r_pad) hm.qh[tid] = 0;
-    if (tid == 0) { hm.inv_tau = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f; hm.l1_sel = l1_sel; }
-    __syncthreads();
     if (idx_r) for (int j = tid; j < r; j += NT) idx_r[(size_t)bh * r + j] = hm.i1[j];
 
     PHASE_MARK(0);
@@ -142,8 +157,18 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         return;
     }
 
-    // ------------------------------------------------------------------ a2: stream r rows of Kt
     const sparq_half* Kt_head = Kt + kv_head * (size_t)D * S_max;
+    uint32_t kmax = 0, kabs_bits = 0;
+    if constexpr (FROM_SCRATCH) {
+        // ---------------------------------------------------------------- a2 was done by the split kernel
+        const uint4* src = reinterpret_cast<const uint4*>(ws_keys + (size_t)bh * S_max);
+        for (int i = tid; i < (n + 3) / 4; i += NT) reinterpret_cast<uint4*>(keys)[i] = src[i];
+        for (int p = tid; p < splits; p += NT) {
+            kmax = max(kmax, ws_part[((size_t)bh * splits + p) * 2]);
+            kabs_bits = max(kabs_bits, ws_part[((size_t)bh * splits + p) * 2 + 1]);
+        }
+    } else {
+    // ------------------------------------------------------------------ a2: stream r rows of Kt
     const int n8 = (n + 7) & ~7;                             // whole 16-byte vectors; n8 <= S_max
     const int n_chunks = (n8 + CH - 1) / CH;
     const int nb = r_pad / RB;
@@ -162,7 +187,6 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     };
     if (warp == 0) for (int it = 0; it < min(STAGES, total); ++it) issue(it, it);
 
-    uint32_t kmax = 0;
     __half2 mx[4];                                           // largest |K| among the valid streamed values
 #pragma unroll
     for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
@@ -204,7 +228,8 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         return;
     }
     PHASE_MARK(1);
-    uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
+    kabs_bits = __float_as_uint(mx_to_float(mx));
+    }
     group_max2_u32<CTA>(kmax, kabs_bits, sh.redu, tid);      // barriers: keys complete, ring is dead
 
     // ------------------------------------------------------------------ a3-a6 (scratch in the dead ring)
@@ -215,6 +240,75 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     finish<CTA, 8>(tid, hm, keys, kmax, sel_res, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
                    vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
     PHASE_MARK(2);
+}
+
+// ---------------------------------------------------------------------------------- split-S plan
+// When there are fewer (batch, head) units than SMs (batch-1 decode over a long cache), one CTA
+// per unit leaves most of the GPU idle.  The split plan cuts every unit's sequence into `splits`
+// slices: grid (splits, units), 128 threads, each CTA repeats a1 (cheap) and streams its slice of
+// the r selected Kt rows with plain 128-bit loads (8 rows in flight per thread), writing the
+// slice's keys to a scratch buffer and its largest key / largest |K| beside them.  The second
+// kernel, sparq_decode_kernel<true>, one CTA per unit, picks the keys up and runs a3-a6 unchanged,
+// so the selected set is exactly the one of the unsplit plans.
+constexpr int SNT = 128;                 // threads of a scores CTA
+constexpr int SCH = SNT * 8;             // positions a scores CTA covers per pass
+using SCTA = Group<SNT, 0>;
+
+__global__ void __launch_bounds__(SNT)
+sparq_split_scores_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ Kt,
+                          const int32_t* __restrict__ seq_lens, int Hq, int Hkv, int S_max, int r, int k, int splits,
+                          uint32_t* __restrict__ ws_keys, uint32_t* __restrict__ ws_part, int32_t* __restrict__ idx_r) {
+    __shared__ HeadMeta hm;
+    __shared__ float red[2 * SCTA::NW];
+    __shared__ uint32_t redu[2 * SCTA::NW];
+    __shared__ uint32_t cnt[4];
+    const int tid = threadIdx.x, p = blockIdx.x, bh = blockIdx.y;
+    const int b = bh / Hq, h = bh % Hq, hkv = h / (Hq / Hkv);
+    const int n = seq_lens[b];
+    uint32_t kmax = 0;
+    __half2 mx[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
+    if (n >= 1 && n <= S_max && k > 0) {                     // otherwise the second kernel reports / returns v_bar
+        top_r_block<SCTA, 8>(tid, q + (size_t)bh * D, r, hm, red, cnt);
+        if (p == 0 && idx_r) for (int j = tid; j < r; j += SNT) idx_r[(size_t)bh * r + j] = hm.i1[j];
+        const uint4* Kt_vec = reinterpret_cast<const uint4*>(Kt + ((size_t)b * Hkv + hkv) * (size_t)D * S_max);
+        const int row_vecs = S_max >> 3;
+        const int n_pass = ((n + 7) / 8 + SNT - 1) / SNT;    // passes of SCH positions over the whole sequence
+        uint32_t* keys = ws_keys + (size_t)bh * S_max;
+        for (int c = p; c < n_pass; c += splits) {           // this CTA's passes: c = p, p + splits, ...
+            const int t0 = c * SCH + tid * 8;
+            const int nvalid = min(8, n - t0);
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            if (nvalid > 0) {
+                uint32_t msk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
+                for (int jb = 0; jb < r; jb += 8) {
+                    uint4 v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = ld_stream(Kt_vec + (size_t)hm.i1[min(jb + u, r - 1)] * row_vecs + (t0 >> 3));
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (jb + u < r) {
+                            v[u].x &= msk[0]; v[u].y &= msk[1]; v[u].z &= msk[2]; v[u].w &= msk[3];
+                            row_fma(acc, mx, v[u], hm.qh[jb + u]);
+                        }
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (e < nvalid) { const uint32_t kk = key32(acc[e]); keys[t0 + e] = kk; kmax = max(kmax, kk); }
+            }
+        }
+    }
+    else if (p == 0 && idx_r && (n < 1 || n > S_max)) {
+        for (int j = tid; j < r; j += SNT) idx_r[(size_t)bh * r + j] = -1;
+    }
+    uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
+    group_max2_u32<SCTA>(kmax, kabs_bits, redu, tid);
+    if (tid == 0) { ws_part[((size_t)bh * splits + p) * 2] = kmax; ws_part[((size_t)bh * splits + p) * 2 + 1] = kabs_bits; }
 }
 
 }  // namespace
@@ -237,10 +331,41 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
                                 int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                 int32_t* status, cudaStream_t stream) {
     const size_t dyn = decode_dynamic_smem(S_max);
-    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
-    sparq_decode_kernel<<<B * Hq, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, idx_r,
-                                                     idx_k, alpha, status);
+    sparq_decode_kernel<false><<<B * Hq, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, idx_r,
+                                                            idx_k, alpha, status, nullptr, nullptr, 0);
+    return cudaGetLastError();
+}
+
+// Slices per unit of the split plan: enough CTAs for about two per SM, at least one pass of SCH
+// positions per slice; 0 when the plan does not apply (as many units as SMs, or a short cache).
+int split_count(int units, int S_max, int n_sm) {
+    if (n_sm <= 0 || units >= n_sm || S_max < 2 * SCH) return 0;
+    const int want = (2 * n_sm + units - 1) / units;
+    const int cap = (S_max + SCH - 1) / SCH;
+    const int s = want < cap ? want : cap;
+    return s < 2 ? 0 : s;
+}
+
+size_t split_scratch_bytes(int units, int S_max, int splits) {
+    return ((size_t)units * S_max + (size_t)units * splits * 2) * sizeof(uint32_t);
+}
+
+cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
+                                      int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                      int32_t* status, int splits, void* scratch, cudaStream_t stream) {
+    const int units = B * Hq;
+    uint32_t* ws_keys = static_cast<uint32_t*>(scratch);
+    uint32_t* ws_part = ws_keys + (size_t)units * S_max;
+    const size_t dyn = decode_dynamic_smem(S_max);
+    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    if (e != cudaSuccess) return e;
+    sparq_split_scores_kernel<<<dim3(splits, units), SNT, 0, stream>>>(q, Kt, seq_lens, Hq, Hkv, S_max, r, k, splits,
+                                                                       ws_keys, ws_part, idx_r);
+    sparq_decode_kernel<true><<<units, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, nullptr,
+                                                          idx_k, alpha, status, ws_keys, ws_part, splits);
     return cudaGetLastError();
 }
 

@@ -224,6 +224,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
         uint32_t* hist1 = hist1_all + kb * FBINS;
         CLK_BEGIN(t_unit);
+#ifdef SPARQ_PHASE_CLOCKS
+        long long ring_wait = 0;
+#endif
         if (gtid < 32) wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
         CLK_BEGIN(t_kf);
         group_wait<SG, 100>(gtid, &sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
@@ -243,7 +246,13 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 const int t0 = c * CH + gtid * 8;
                 const int nvalid = min(8, n - t0);           // positions of this thread's vector inside the sequence
                 for (int jb = 0; jb < r; jb += RB) {
+#ifdef SPARQ_PHASE_CLOCKS
+                    const long long t_f0 = clock64();
+#endif
                     wait_or_abort<20>(&sh.full[s], parity, sh, a.status);
+#ifdef SPARQ_PHASE_CLOCKS
+                    ring_wait += clock64() - t_f0;
+#endif
                     stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid, hm.qh + jb, r - jb,
                                           nvalid);
                     __syncwarp();
@@ -271,6 +280,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         SG::sync();                                          // every key of the unit is written
         if (gtid == 0) mbar_arrive(&sh.keys_full[kb]);
         CLK_ADD(4, t_unit, gtid == 0);
+#ifdef SPARQ_PHASE_CLOCKS
+        if (gtid == 0) atomicAdd(&g_pipe_clocks[3], (unsigned long long)ring_wait);
+#endif
     }
 }
 

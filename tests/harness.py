@@ -4,6 +4,9 @@ own entry points, run the oracle on the same fp16 inputs, and compare under the 
 2e-3 max-abs and 1e-3 relative L2)."""
 from __future__ import annotations
 
+import contextlib
+import os
+
 import numpy as np
 import torch
 
@@ -14,6 +17,23 @@ MAX_ABS = 2e-3      # fp16 caches, fp16 output
 REL_L2 = 1e-3
 GAP_WAIVER = 1e-6   # relative gap between the last selected and first rejected value
 ALPHA_TOL = 5e-5    # fp32 exponentials of fp32-rounded logits against the float64 alpha
+
+
+@contextlib.contextmanager
+def decode_plan(name):
+    """Force one of the sparq_decode plans ('simple', 'pipe', 'split') or None for the library's choice."""
+    old = os.environ.get("SPARQ_DECODE_PLAN")
+    if name is None:
+        os.environ.pop("SPARQ_DECODE_PLAN", None)
+    else:
+        os.environ["SPARQ_DECODE_PLAN"] = name
+    try:
+        yield
+    finally:
+        if old is None:
+            os.environ.pop("SPARQ_DECODE_PLAN", None)
+        else:
+            os.environ["SPARQ_DECODE_PLAN"] = old
 
 
 class DeviceCache:
@@ -48,8 +68,11 @@ class DeviceCache:
         idx_r = torch.full((B, Hq, r), -7, dtype=torch.int32, device=q.device)
         idx_k = torch.full((B, Hq, max(k, 1)), -7, dtype=torch.int32, device=q.device)[:, :, :k].contiguous()
         alpha = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=q.device)
+        # a workspace whenever the library says one helps: few units over a long cache then take the split-S plan
+        nbytes = sparq.sparq_workspace_bytes(B, Hq, self.Hkv, d, self.S_max, r, k)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=q.device) if nbytes else None
         sparq.sparq_decode(q, self.K, self.Kt, self.V, self.vbar, self.seq_lens, r, k, out, idx_r=idx_r,
-                           idx_k=idx_k if k > 0 else None, alpha=alpha, status=self.status)
+                           idx_k=idx_k if k > 0 else None, alpha=alpha, workspace=ws, status=self.status)
         torch.cuda.synchronize()
         return dict(out=out.cpu().numpy().astype(np.float64), i1=idx_r.cpu().numpy(), i2=idx_k.cpu().numpy(),
                     alpha=alpha.cpu().numpy().astype(np.float64))

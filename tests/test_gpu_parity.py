@@ -38,10 +38,37 @@ def test_c0_tiny_single_step_against_numpy_oracle():
     _dense_check(c, cache, c.q_steps[0], "c0")
 
 
-def test_c1_llama2_batch1_all_heads():
+@pytest.mark.parametrize("plan", ["split", "pipe", "simple"])
+def test_c1_llama2_batch1_all_heads(plan):
+    """Batch 1, 32 heads: fewer units than SMs, so the library's own choice is the split-S plan;
+    the two single-kernel plans must give the same parity."""
     c = synth.make_case("c1")
-    waived, total = H.run_case_all_heads(c, "c1")
+    assert sparq.sparq_workspace_bytes(1, 32, 32, 128, 4096, 32, 128) > 0
+    with H.decode_plan(plan):
+        waived, total = H.run_case_all_heads(c, "c1 " + plan)
     assert total == 32 and waived <= 1
+
+
+def test_split_plan_long_ragged_gqa_and_bad_length():
+    """Split-S over long ragged GQA sequences (slices end inside 16-byte vectors), an invalid
+    sequence among them, and the same call without a workspace giving identical results."""
+    c = synth.make_case("c4", B=3, Hq=8, Hkv=2, ragged=(9000, 20000), n_steps=1, backend="numpy")
+    with H.decode_plan("split"):
+        waived, total = H.run_case_all_heads(c, "split ragged")
+    assert total == 24 and waived <= 1
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
+    q = c.q_steps[0]
+    a = cache.decode(q, c.r, c.k)                                   # library's choice: split (24 units)
+    with H.decode_plan("simple"):
+        b = cache.decode(q, c.r, c.k)
+    for key in a:
+        np.testing.assert_array_equal(a[key], b[key])
+    cache.seq_lens[1] = 0
+    with H.decode_plan("split"):
+        bad = cache.decode(q, c.r, c.k)
+    cache.check_status(sparq.DEV_BAD_SEQ_LEN)
+    assert (bad["out"][1] == 0).all() and (bad["i1"][1] == -1).all() and (bad["i2"][1] == -1).all()
+    np.testing.assert_array_equal(bad["out"][0], a["out"][0])
 
 
 @pytest.mark.parametrize("name,kw", [
