@@ -91,8 +91,11 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
 size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
     (void)r; (void)k;
     if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
-    const int splits = split_count(B * Hq, S_max, device_sm_count());
-    return splits ? split_scratch_bytes(B * Hq, S_max, splits) : 0;
+    // worth having: fewer units than SMs (slicing), or keys too long for the pipelined kernel
+    const int n_sm = device_sm_count();
+    const int splits = split_count(B * Hq, S_max, n_sm);
+    if (!splits || (B * Hq >= n_sm && pipe_fits(S_max, device_smem_optin()))) return 0;
+    return split_scratch_bytes(B * Hq, S_max, splits);
 }
 
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -105,10 +108,12 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
     if (S_max > sparq_max_seq_len()) return SPARQ_ERR_TOO_LONG;
     const int plan = forced_plan();
-    const int splits = split_count(B * Hq, S_max, device_sm_count());
+    const int n_sm = device_sm_count();
+    const int splits = split_count(B * Hq, S_max, n_sm);
     const bool ws_ok = splits && workspace && workspace_bytes >= split_scratch_bytes(B * Hq, S_max, splits);
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
-    if (ws_ok && (plan == 0 || plan == 3))
+    const bool split_pays = B * Hq < n_sm || !pipe_fits(S_max, device_smem_optin());
+    if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
         return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
                                             alpha, status, splits, workspace, (cudaStream_t)stream));
     const bool fits = pipe_fits(S_max, device_smem_optin());

@@ -27,6 +27,7 @@ constexpr int BM_WORDS = 2048;           // bitmap capacity: 65536 positions
 using CTA = Group<NT, 0>;
 
 static_assert(post_scratch_bytes(CTA::NHW, BM_WORDS) <= RING_BYTES, "post-phase scratch must fit the dead ring");
+constexpr int SCRATCH_ONLY_BYTES = (int)((post_scratch_bytes(CTA::NHW, BM_WORDS) + 127) & ~(size_t)127);
 static_assert(RB <= 8, "HeadMeta::qh padding");
 
 
@@ -120,7 +121,8 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                     const uint32_t* __restrict__ ws_keys, const uint32_t* __restrict__ ws_part, int splits) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;                                       // a2: STAGES x [RB rows x CH positions] fp16
-    uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);  // [n] approximate-score keys
+    // [n] approximate-score keys, after the ring (or, without a2, after the post-phase scratch alone)
+    uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + (FROM_SCRATCH ? SCRATCH_ONLY_BYTES : RING_BYTES));
     __shared__ DecodeShared sh;
     HeadMeta& hm = sh.hm;
 
@@ -324,6 +326,7 @@ extern "C" int sparq_debug_phase_clocks(unsigned long long* out16, int reset) {
 
 size_t decode_static_smem() { return sizeof(DecodeShared); }
 size_t decode_dynamic_smem(int S_max) { return (size_t)RING_BYTES + (size_t)S_max * sizeof(uint32_t); }
+static size_t decode_dynamic_smem_from_scratch(int S_max) { return (size_t)SCRATCH_ONLY_BYTES + (size_t)S_max * sizeof(uint32_t); }
 int decode_max_positions() { return BM_WORDS * 32; }
 
 cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -339,13 +342,17 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
 }
 
 // Slices per unit of the split plan: enough CTAs for about two per SM, at least one pass of SCH
-// positions per slice; 0 when the plan does not apply (as many units as SMs, or a short cache).
+// positions per slice; 0 when the plan does not apply (a short cache).  With at least as many
+// units as SMs the answer is 1: no slicing, but still two kernels -- a pure streaming kernel at
+// high occupancy, then the latency-bound stages with the keys read back from the workspace --
+// which pays off when the keys of one unit fill most of an SM's shared memory.
 int split_count(int units, int S_max, int n_sm) {
-    if (n_sm <= 0 || units >= n_sm || S_max < 2 * SCH) return 0;
+    if (n_sm <= 0 || S_max < 2 * SCH) return 0;
+    if (units >= n_sm) return 1;
     const int want = (2 * n_sm + units - 1) / units;
     const int cap = (S_max + SCH - 1) / SCH;
     const int s = want < cap ? want : cap;
-    return s < 2 ? 0 : s;
+    return s < 1 ? 1 : s;
 }
 
 size_t split_scratch_bytes(int units, int S_max, int splits) {
@@ -359,7 +366,7 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
     const int units = B * Hq;
     uint32_t* ws_keys = static_cast<uint32_t*>(scratch);
     uint32_t* ws_part = ws_keys + (size_t)units * S_max;
-    const size_t dyn = decode_dynamic_smem(S_max);
+    const size_t dyn = decode_dynamic_smem_from_scratch(S_max);
     cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     sparq_split_scores_kernel<<<dim3(splits, units), SNT, 0, stream>>>(q, Kt, seq_lens, Hq, Hkv, S_max, r, k, splits,
