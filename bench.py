@@ -37,7 +37,7 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 683.6e6   # 2 x (336.44 + 5.37) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md
 
 
 def compulsory_bytes_per_unit(n: float, r: int, k: int, d: int) -> float:
