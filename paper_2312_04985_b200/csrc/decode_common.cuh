@@ -56,16 +56,22 @@ struct PostScratch {
     uint32_t* res;                // [4]
     uint32_t* band;               // [4]
 };
-// bytes of the scratch that may alias a dead buffer (everything except i2 and the small arrays)
+// Bytes of the scratch that may alias a dead buffer (everything except i2 and the small arrays).
+// The half-warp merge area of stage a5 reuses the select stage's histogram/list and the head of
+// the bitmaps, all dead by then, so it costs no space of its own.
 __host__ __device__ constexpr size_t post_scratch_bytes(int nhw, int bm_words) {
-    return (size_t)HIST_BINS * 4 + 2 * (size_t)bm_words * 4 + (size_t)nhw * (D + 2) * 4 + (size_t)CAND_MAX * 12;
+    const size_t select_part = (size_t)HIST_BINS * 4 + 2 * (size_t)bm_words * 4;
+    const size_t merge_part = (size_t)nhw * (D + 2) * 4;
+    return (((select_part > merge_part ? select_part : merge_part) + 7) & ~(size_t)7) + (size_t)CAND_MAX * 12;
 }
 __device__ __forceinline__ void carve_post_scratch(PostScratch& sc, unsigned char* base, int nhw, int bm_words) {
+    const size_t select_part = (size_t)HIST_BINS * 4 + 2 * (size_t)bm_words * 4;
+    const size_t merge_part = (size_t)nhw * (D + 2) * 4;
     sc.hist = reinterpret_cast<uint32_t*>(base);
     sc.bm_sel = sc.hist + HIST_BINS;
     sc.bm_tie = sc.bm_sel + bm_words;
-    sc.merge = reinterpret_cast<float*>(sc.bm_tie + bm_words);
-    sc.cand_val = reinterpret_cast<unsigned long long*>(sc.merge + nhw * (D + 2));
+    sc.merge = reinterpret_cast<float*>(base);               // live only after the index list is built
+    sc.cand_val = reinterpret_cast<unsigned long long*>(base + (((select_part > merge_part ? select_part : merge_part) + 7) & ~(size_t)7));
     sc.cand_pos = reinterpret_cast<int32_t*>(sc.cand_val + CAND_MAX);
 }
 
@@ -106,21 +112,27 @@ template <int RB, int CH8>
 __device__ __forceinline__ void stage_fma(float (&acc)[8], __half2 (&mx)[4], const uint4* src, const uint16_t* qh_jb,
                                           int rows_left, int nvalid) {
     static_assert(RB == 4 || RB == 8, "query components are fetched as one 8- or 16-byte vector");
-    if (nvalid >= 8 && rows_left >= RB) {                    // the common case: no predicates at all
+    // One decision per warp, so that a warp never runs both variants one after the other.
+    const bool plain = __all_sync(FULL, nvalid >= 8) && rows_left >= RB;
+    if (plain) {                                             // the common case: no predicates at all
         uint32_t qw[RB / 2];
         if constexpr (RB == 8) { const uint4 q8 = *reinterpret_cast<const uint4*>(qh_jb); qw[0] = q8.x; qw[1] = q8.y; qw[2] = q8.z; qw[3] = q8.w; }
         else { const uint2 q4 = *reinterpret_cast<const uint2*>(qh_jb); qw[0] = q4.x; qw[1] = q4.y; }
 #pragma unroll
         for (int u = 0; u < RB; ++u)
             row_fma(acc, mx, src[u * CH8], (uint16_t)((u & 1) ? (qw[u >> 1] >> 16) : (qw[u >> 1] & 0xffffu)));
-    } else if (nvalid > 0) {
+    } else {
+        // the warp that holds the end of the sequence, or the last, partial batch of rows
         uint32_t msk[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
-        for (int u = 0; u < RB && u < rows_left; ++u) {      // padded rows were not copied
-            uint4 v = src[u * CH8];
-            v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
-            row_fma(acc, mx, v, qh_jb[u]);
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+            if (u < rows_left) {                             // uniform; padded rows were not copied
+                uint4 v = src[u * CH8];
+                v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
+                row_fma(acc, mx, v, qh_jb[u]);
+            }
         }
     }
 }
