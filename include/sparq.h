@@ -108,11 +108,14 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
  *   rounded to fp16 (Eq. (10)).  k == 0 gives out = vbar.
  * Optional outputs (each may be NULL): idx_r [B,Hq,r] int32 = i1 ascending; idx_k [B,Hq,k]
  * int32 = i2 ascending, unused tail -1; alpha [B,Hq] fp32.
- * workspace: optional device scratch for the split-S plan.  When there are fewer (batch, head)
- * units than SMs (batch-1 decode over a long cache) sparq_workspace_bytes() is non-zero, and a
- * workspace of that size lets the call cut every sequence into slices handled by different thread
- * blocks (same results, far lower latency).  With workspace NULL or too small, or when
- * sparq_workspace_bytes() is 0, a single-kernel plan is used.  Contents are undefined afterwards.
+ * workspace: optional device scratch; sparq_workspace_bytes() says how much helps for the given
+ * shapes (0: none).  Three uses, results identical in all of them: fewer (batch, head) units
+ * than SMs -- every sequence is cut into slices handled by different thread blocks (far lower
+ * latency for batch-1 decode over a long cache); a cache too long for the persistent kernel -- the
+ * scores take a streaming kernel of their own; more units than SMs on the persistent kernel -- 64
+ * bytes for a counter from which the thread blocks draw their units, which evens out their
+ * finishing times.  With workspace NULL or too small a plan without scratch is used.  The call
+ * clears what it needs; contents are undefined afterwards.
  */
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                  const sparq_half* vbar, const int32_t* seq_lens,

@@ -40,6 +40,8 @@ int forced_plan() {
     return 0;
 }
 
+constexpr size_t SPARQ_PIPE_WORKSPACE_BYTES = 64;
+
 int rc(cudaError_t e) { return e == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA; }
 
 }  // namespace
@@ -94,8 +96,9 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     // worth having: fewer units than SMs (slicing), or keys too long for the pipelined kernel
     const int n_sm = device_sm_count();
     const int splits = split_count(B * Hq, S_max, n_sm);
-    if (!splits || (B * Hq >= n_sm && pipe_fits(S_max, device_smem_optin()))) return 0;
-    return split_scratch_bytes(B * Hq, S_max, splits);
+    if (pipe_fits(S_max, device_smem_optin()) && (B * Hq >= n_sm || !splits))
+        return B * Hq > n_sm ? SPARQ_PIPE_WORKSPACE_BYTES : 0;   // the persistent kernel's unit counter
+    return splits ? split_scratch_bytes(B * Hq, S_max, splits) : 0;
 }
 
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -118,9 +121,13 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
                                             alpha, status, splits, workspace, (cudaStream_t)stream));
     const bool fits = pipe_fits(S_max, device_smem_optin());
     if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
-    if (fits && plan != 1)
+    if (fits && plan != 1) {
+        // with a workspace the persistent CTAs draw their units from a counter instead of a fixed share
+        unsigned int* counter = (workspace && workspace_bytes >= SPARQ_PIPE_WORKSPACE_BYTES && B * Hq > n_sm)
+                                    ? static_cast<unsigned int*>(workspace) : nullptr;
         return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
-                                           alpha, status, device_sm_count(), (cudaStream_t)stream));
+                                           alpha, status, n_sm, counter, (cudaStream_t)stream));
+    }
     return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
                                   status, (cudaStream_t)stream));
 }
@@ -154,7 +161,7 @@ int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_ha
 
 size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d) {
     if (B < 1 || Hq < 1 || Hkv < 1 || d < 1) return 0;
-    return ((size_t)2 * B * Hq * d + (size_t)2 * B * Hkv * d) * sizeof(sparq_half);
+    return ((size_t)2 * B * Hq * d + (size_t)2 * B * Hkv * d) * sizeof(sparq_half) + SPARQ_PIPE_WORKSPACE_BYTES;
 }
 
 int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, const sparq_half* v_new_host,
@@ -176,8 +183,9 @@ int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, cons
         return SPARQ_ERR_CUDA;
     int code = sparq_cache_append(k_dev, v_dev, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, d, S_max, status, stream);
     if (code != SPARQ_OK) return code;
+    void* ws = v_dev + nkv;                                  // the tail of the staging area: the decode's small workspace
     code = sparq_decode(q_dev, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, out_dev, nullptr, nullptr, nullptr,
-                        nullptr, 0, status, stream);
+                        ws, SPARQ_PIPE_WORKSPACE_BYTES, status, stream);
     if (code != SPARQ_OK) return code;
     if (cudaMemcpyAsync(out_host, out_dev, nq * sizeof(sparq_half), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return SPARQ_ERR_CUDA;

@@ -31,7 +31,7 @@ bool pipe_fits(int S_max, int smem_optin);
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, int n_sm, cudaStream_t stream);
+                                     int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream);
 
 // dense_decode.cu
 int dense_splits(int B, int Hkv, int S_max);

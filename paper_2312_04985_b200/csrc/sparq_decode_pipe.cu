@@ -43,6 +43,8 @@ static_assert(RB <= 8, "HeadMeta::qh padding");
 // [2] stream waiting for a free key buffer, [3] stream waiting for ring data, [4] stream total per unit,
 // [5] producer waiting for a free ring slot, [6] producer a1
 #ifdef SPARQ_PHASE_CLOCKS
+__device__ unsigned long long g_cta_end[256];
+__device__ unsigned long long g_cta_begin[256];
 __device__ unsigned long long g_pipe_clocks[16];
 #define CLK_BEGIN(var) long long var = clock64()
 #define CLK_ADD(i, var, cond) do { if (cond) atomicAdd(&g_pipe_clocks[i], (unsigned long long)(clock64() - var)); } while (0)
@@ -75,6 +77,7 @@ struct Args {
     int32_t *idx_r, *idx_k;
     float* alpha;
     int32_t* status;
+    unsigned int* unit_counter;   // zeroed device word for dynamic unit assignment, or NULL: static stride
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -105,18 +108,40 @@ __device__ __forceinline__ void group_wait(int gtid, uint64_t* bar, uint32_t par
 }
 
 // ---------------------------------------------------------------------------------- a1 warp
-__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_mine) {
+// Units are handed out first come, first served when a zeroed counter is available (CTAs differ by
+// 10-20 % in how fast they get through a unit, so a fixed share per CTA leaves the last ones
+// running alone); without a counter CTA i takes units i, i + gridDim.x, ...  After the last unit
+// the a1 warp publishes NPOST end markers (bh = -1), one for each post group.
+__device__ __forceinline__ int next_unit(const Args& a, int bh, int lane) {
+    int u = bh + (int)gridDim.x;
+    if (a.unit_counter) {
+        if (lane == 0) u = (int)gridDim.x + (int)atomicAdd(a.unit_counter, 1u);
+        u = __shfl_sync(FULL, u, 0);
+    }
+    return u < a.n_units ? u : -1;
+}
+
+__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
     const int lane = threadIdx.x & 31;
+    int bh = (int)blockIdx.x < a.n_units ? (int)blockIdx.x : -1;
     uint2 qraw = make_uint2(0, 0);                           // components 4*lane .. 4*lane+3 of the unit's q
     int n_next = 0;
-    if (n_mine > 0) {
-        qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)blockIdx.x * D + lane * 4);
-        n_next = a.seq_lens[blockIdx.x / a.Hq];
+    if (bh >= 0) {
+        qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + lane * 4);
+        n_next = a.seq_lens[bh / a.Hq];
     }
-    for (int j = 0; j < n_mine; ++j) {
-        const int bh = blockIdx.x + j * gridDim.x;
+    int markers = 0;
+    for (int j = 0; markers < NPOST; ++j) {
         const int m = j % NMETA;
         HeadMeta& hm = sh.meta[m];
+        if (bh < 0) {                                        // no unit left: an end marker for one post group
+            wait_or_abort<200>(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
+            if (lane == 0) { hm.bh = -1; hm.n = 0; hm.k_eff = 0; hm.valid = 0; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.meta_full[m]);
+            ++markers;
+            continue;
+        }
         // key = |q_c| bits above (127 - c): distinct keys, larger |q| first, then smaller c
         const int n = n_next;
         const bool valid = n >= 1 && n <= a.S_max;
@@ -124,9 +149,10 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_min
         const uint16_t hb[4] = {(uint16_t)(qraw.x & 0xffffu), (uint16_t)(qraw.x >> 16), (uint16_t)(qraw.y & 0xffffu),
                                 (uint16_t)(qraw.y >> 16)};
         // the next unit's query and length travel while this unit is ranked
-        if (j + 1 < n_mine) {
-            qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)(bh + gridDim.x) * D + lane * 4);
-            n_next = a.seq_lens[(bh + gridDim.x) / a.Hq];
+        const int bh_next = next_unit(a, bh, lane);
+        if (bh_next >= 0) {
+            qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh_next * D + lane * 4);
+            n_next = a.seq_lens[bh_next / a.Hq];
         }
         wait_or_abort<200>(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
         CLK_BEGIN(t_a1);
@@ -176,18 +202,20 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, int n_min
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.meta_full[m]);
         CLK_ADD(6, t_a1, lane == 0);
+        bh = bh_next;
     }
 }
 
 // ---------------------------------------------------------------------------------- producer
-__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int n_mine, int p) {
+__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int p) {
     const int lane = threadIdx.x & 31;
     const int g_heads = a.Hq / a.Hkv;
     uint32_t g = 0;                                          // ring stages issued so far
-    for (int j = 0; j < n_mine; ++j) {
+    for (int j = 0, markers = 0; markers < NPOST; ++j) {
         const int m = j % NMETA;
         const HeadMeta& hm = sh.meta[m];
         wait_or_abort<100>(&sh.meta_full[m], ((uint32_t)(j / NMETA)) & 1u, sh, a.status);
+        if (hm.bh < 0 || sh.abort_flag) { ++markers; continue; }
         // the unit's ring stages: [chunk c][row batch jb] -> RB rows x CH positions
         if (hm.k_eff > 0) {
             const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq, n = hm.n;
@@ -214,11 +242,11 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
 
 // ---------------------------------------------------------------------------------- stream group
 __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
-                                            uint32_t* hist1_all, int n_mine) {
+                                            uint32_t* hist1_all) {
     const int gtid = threadIdx.x - LEAD, lane = gtid & 31;
     int s = 0;                                               // ring slot and its phase parity
     uint32_t parity = 0;
-    for (int j = 0; j < n_mine; ++j) {
+    for (int j = 0, markers = 0; markers < NPOST; ++j) {
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
@@ -232,6 +260,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         group_wait<SG, 100>(gtid, &sh.keys_free[kb], (((uint32_t)(j / NKB)) & 1u) ^ 1u, sh, a.status);
         CLK_ADD(2, t_kf, gtid == 0);
         const int n = hm.n, r = a.r;
+        if (hm.bh < 0 || sh.abort_flag) ++markers;           // forwarded to the post group below (group-uniform)
         if (hm.k_eff > 0) {
             uint32_t kmax = 0;
             __half2 mx[4];                                   // largest |K| among the valid streamed values
@@ -289,19 +318,25 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 // ---------------------------------------------------------------------------------- post groups
 template <class PG>
 __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, uint32_t* hist1_all,
-                                          unsigned char* scratch, int n_mine, int p) {
+                                          unsigned char* scratch, int p) {
     const int gtid = threadIdx.x - LEAD - SNT - p * GNT;
     PostScratch sc;
     carve_post_scratch(sc, scratch, PG::NHW, a.S_cap / 32);
     sc.i2 = sh.i2[p]; sc.red = sh.red[p]; sc.redu = sh.redu[p]; sc.res = sh.res[p]; sc.band = sh.band[p];
     const int g_heads = a.Hq / a.Hkv;
-    for (int j = p; j < n_mine; j += NPOST) {
+    for (int j = p;; j += NPOST) {
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
         CLK_BEGIN(t_w);
         group_wait<PG, 100>(gtid, &sh.keys_full[kb], ((uint32_t)(j / NKB)) & 1u, sh, a.status);
         CLK_ADD(1, t_w, gtid == 0);
         CLK_BEGIN(t_p);
+        if (hm.bh < 0 || sh.abort_flag) {                    // end marker (or a wait gave up): this group is done
+#ifdef SPARQ_PHASE_CLOCKS
+            if (gtid == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); atomicMax(&g_cta_end[blockIdx.x], gt); }
+#endif
+            break;
+        }
         const int bh = hm.bh, b = bh / a.Hq, h = bh % a.Hq;
         const size_t kv_head = (size_t)b * a.Hkv + h / g_heads;
         sparq_half* out_row = a.out + (size_t)bh * D;
@@ -354,13 +389,15 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) 
     }
     for (int i = threadIdx.x; i < NKB * FBINS; i += NT) hist1_all[i] = 0;
     __syncthreads();
-    const int n_mine = (a.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // units blockIdx.x + j*gridDim.x
+#ifdef SPARQ_PHASE_CLOCKS
+    if (threadIdx.x == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_cta_begin[blockIdx.x] = gt; g_cta_end[blockIdx.x] = 0; }
+#endif
     const int warp = threadIdx.x >> 5;
-    if (warp < NPROD) producer_role(a, sh, ring, n_mine, warp);
-    else if (warp == NPROD) a1_role(a, sh, n_mine);
-    else if (warp < LEAD / 32 + SNT / 32) stream_role(a, sh, ring, keys_all, hist1_all, n_mine);
-    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, hist1_all, scratch0, n_mine, 0);
-    else post_role<PG1>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, n_mine, 1);
+    if (warp < NPROD) producer_role(a, sh, ring, warp);
+    else if (warp == NPROD) a1_role(a, sh);
+    else if (warp < LEAD / 32 + SNT / 32) stream_role(a, sh, ring, keys_all, hist1_all);
+    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0>(a, sh, keys_all, hist1_all, scratch0, 0);
+    else post_role<PG1>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1);
 }
 
 size_t pipe_dynamic_smem(int S_cap) {
@@ -375,6 +412,12 @@ extern "C" int sparq_debug_pipe_clocks(unsigned long long* out16, int reset) {
     cudaDeviceSynchronize();
     if (out16 && cudaMemcpyFromSymbol(out16, g_pipe_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
     if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_pipe_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+extern "C" int sparq_debug_cta_times(unsigned long long* begin256, unsigned long long* end256) {
+    cudaDeviceSynchronize();
+    if (cudaMemcpyFromSymbol(begin256, g_cta_begin, sizeof(unsigned long long) * 256) != cudaSuccess) return 1;
+    if (cudaMemcpyFromSymbol(end256, g_cta_end, sizeof(unsigned long long) * 256) != cudaSuccess) return 1;
     return 0;
 }
 extern "C" int sparq_debug_post_clocks(unsigned long long* out16, int reset) {
@@ -395,15 +438,19 @@ bool pipe_fits(int S_max, int smem_optin) {
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, int n_sm, cudaStream_t stream) {
+                                     int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream) {
     Args a;
     a.q = q; a.K = K; a.Kt = Kt; a.V = V; a.vbar = vbar; a.seq_lens = seq_lens;
     a.n_units = B * Hq; a.Hq = Hq; a.Hkv = Hkv; a.S_max = S_max; a.S_cap = pipe_s_cap(S_max); a.r = r; a.k = k;
-    a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status;
+    a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status; a.unit_counter = unit_counter;
     const size_t dyn = pipe_dynamic_smem(a.S_cap);
     cudaError_t e = cudaFuncSetAttribute(sparq_decode_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     const int grid = a.n_units < n_sm ? a.n_units : n_sm;
+    if (unit_counter) {
+        e = cudaMemsetAsync(unit_counter, 0, sizeof(unsigned int), stream);
+        if (e != cudaSuccess) return e;
+    }
     sparq_decode_pipe_kernel<<<grid, NT, dyn, stream>>>(a);
     return cudaGetLastError();
 }
