@@ -28,8 +28,8 @@ constexpr int NPROD = 2;                 // producer warps (one warp alone canno
 constexpr int LEAD = 32 * (NPROD + 1);   // producer warps + a1 warp
 constexpr int NT = LEAD + SNT + NPOST * GNT;
 constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
-constexpr int RB = 4;                    // Kt rows per ring stage
-constexpr int STAGES = 7;
+constexpr int RB = 8;                    // Kt rows per ring stage (32 KB stages: fewer hand-offs beat a deeper ring, measured)
+constexpr int STAGES = 3;
 constexpr int STAGE_BYTES = RB * CH * 2;
 constexpr int RING_BYTES = STAGES * STAGE_BYTES;
 constexpr int NKB = 3;                   // key buffers: one being written, two being post-processed
