@@ -23,7 +23,11 @@
  *   - Layouts (row-major, innermost last):
  *         q, out        [B, Hq, d]
  *         K, V          [B, Hkv, S_max, d]
- *         Kt            [B, Hkv, d, S_max]
+ *         Kt            [B, Hkv, d, S_max]     with zeros from position seq_lens[b] to the end of
+ *                                              its 16-byte vector (8 positions); sparq_cache_build
+ *                                              and sparq_cache_append keep it so.  Readers take
+ *                                              whole vectors unmasked; finite junk there only
+ *                                              loosens an error bound, non-finite junk is unsupported
  *         vsum (fp32), vbar (fp16), k_new, v_new   [B, Hkv, d]
  *         seq_lens (int32)   [B]     number of valid positions of sequence b
  *     Query head h reads KV head h / (Hq / Hkv): consecutive query heads share a KV head

@@ -19,7 +19,10 @@ cache_append_kernel(const sparq_half* __restrict__ k_new, const sparq_half* __re
     const size_t head = (size_t)bh * S_max * D;
     K[head + (size_t)n * D + c] = kc;
     V[head + (size_t)n * D + c] = vc;
-    Kt[head + (size_t)c * S_max + n] = kc;                    // the small non-contiguous write
+    // the small non-contiguous write.  Invariant of the layout: the rest of the 16-byte vector that
+    // holds the last valid position is zero, so readers may take whole vectors without masking.
+    if ((n & 7) == 0) *reinterpret_cast<uint4*>(Kt + head + (size_t)c * S_max + n) = make_uint4(kc, 0u, 0u, 0u);
+    else Kt[head + (size_t)c * S_max + n] = kc;
     float s = vsum[(size_t)bh * D + c] + __half2float(__ushort_as_half(vc));
     vsum[(size_t)bh * D + c] = s;
     vbar[(size_t)bh * D + c] = __half_as_ushort(__float2half_rn(s / (float)(n + 1)));
@@ -45,9 +48,10 @@ cache_transpose_kernel(const sparq_half* __restrict__ K, sparq_half* __restrict_
         tile[tt][c] = (t0 + tt < n) ? K[head + (size_t)(t0 + tt) * D + c] : (uint16_t)0;
     }
     __syncthreads();
+    const int n8 = (n + 7) & ~7;                               // zero fill up to the end of the last 16-byte vector
     for (int i = tid; i < 64 * D; i += 256) {
         int c = i / 64, tt = i % 64;
-        if (t0 + tt < n) Kt[head + (size_t)c * S_max + t0 + tt] = tile[tt][c];
+        if (t0 + tt < n8) Kt[head + (size_t)c * S_max + t0 + tt] = tile[tt][c];
     }
 }
 

@@ -104,36 +104,26 @@ __device__ __forceinline__ float mx_to_float(const __half2 (&mx)[4]) {
 
 // One ring stage (RB rows of CH8 16-byte vectors each) into a thread's 8 running sums.
 //   src: the thread's vector in row 0 of the stage; qh_jb: the RB query components of these rows
-//   (16-byte aligned); rows_left: selected rows not yet consumed (>= 1); nvalid: how many of the
-//   thread's 8 positions lie inside the sequence.
-// Positions past the sequence end in the straddling vector hold whatever the caller's memory
-// holds; they are masked to zero so that they reach neither a sum nor the |K| maximum.
+//   (16-byte aligned); rows_left: selected rows not yet consumed (>= 1).
+// No masking here.  The Kt layout guarantees zeros between the sequence end and the end of its
+// 16-byte vector, and a thread whose whole vector lies past the end works on whatever the stage
+// holds there; the caller throws that thread's sums and |K| maximum away (it keeps the maximum
+// per chunk for that).
 template <int RB, int CH8>
 __device__ __forceinline__ void stage_fma(float (&acc)[8], __half2 (&mx)[4], const uint4* src, const uint16_t* qh_jb,
-                                          int rows_left, int nvalid) {
+                                          int rows_left) {
     static_assert(RB == 4 || RB == 8, "query components are fetched as one 8- or 16-byte vector");
-    // One decision per warp, so that a warp never runs both variants one after the other.
-    const bool plain = __all_sync(FULL, nvalid >= 8) && rows_left >= RB;
-    if (plain) {                                             // the common case: no predicates at all
+    if (rows_left >= RB) {                                   // uniform; the common case, no predicates at all
         uint32_t qw[RB / 2];
         if constexpr (RB == 8) { const uint4 q8 = *reinterpret_cast<const uint4*>(qh_jb); qw[0] = q8.x; qw[1] = q8.y; qw[2] = q8.z; qw[3] = q8.w; }
         else { const uint2 q4 = *reinterpret_cast<const uint2*>(qh_jb); qw[0] = q4.x; qw[1] = q4.y; }
 #pragma unroll
         for (int u = 0; u < RB; ++u)
             row_fma(acc, mx, src[u * CH8], (uint16_t)((u & 1) ? (qw[u >> 1] >> 16) : (qw[u >> 1] & 0xffffu)));
-    } else {
-        // the warp that holds the end of the sequence, or the last, partial batch of rows
-        uint32_t msk[4];
+    } else {                                                 // the last, partial batch of rows: the rest was not copied
 #pragma unroll
-        for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-            if (u < rows_left) {                             // uniform; padded rows were not copied
-                uint4 v = src[u * CH8];
-                v.x &= msk[0]; v.y &= msk[1]; v.z &= msk[2]; v.w &= msk[3];
-                row_fma(acc, mx, v, qh_jb[u]);
-            }
-        }
+        for (int u = 0; u < RB; ++u)
+            if (u < rows_left) row_fma(acc, mx, src[u * CH8], qh_jb[u]);
     }
 }
 
@@ -397,15 +387,15 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // Returns false (for every thread of the group alike) when the short-cut does not apply -- a warp
 // meets more of the bin's keys than its list segment holds, or the band reaches outside the bin or holds too many keys -- and
 // the caller runs select_generic instead.
+// Z_stream: the softmax denominator relative to the largest key, accumulated by the stream stage.
 template <class G>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
-                                                 float kabs, const PostScratch& sc, uint32_t* hist1, int r, int S_max,
-                                                 const sparq_half* __restrict__ Kt_head, SelectResult& out) {
-    static_assert(G::NT >= 256, "warp 0 scans 256 bins, thread i clears bin i");
+                                                 float kabs, float Z_stream, const PostScratch& sc, uint32_t* hist1, int r,
+                                                 int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out) {
+    static_assert(G::NT >= 256, "thread i clears histogram word i");
     const int lane = gtid & 31, warp = gtid >> 5;
     const int n = hm.n, k_eff = hm.k_eff;
-    const float vmax = unkey32(kmax);
-    const float c1 = hm.inv_tau * LOG2E;
+    (void)kmax;
 
     POST_CLK_INIT();
     if (gtid < 4) sc.band[gtid] = 0;     // [0] band keys below the edge, [1] at/above it, [2] band list length
@@ -421,7 +411,6 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const unsigned lt = (1u << lane) - 1;
 
     const int nwords = (n + 31) >> 5;
-    float zpart = 0.f;
     uint32_t wcount = 0;                                     // this warp's list length (warp-uniform)
     for (int w0 = warp; w0 < nwords; w0 += 4 * G::NW) {      // four words in flight per warp
         uint32_t u[4];
@@ -436,7 +425,6 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         for (int x = 0; x < 4; ++x) {
             const int wi = w0 + x * G::NW;
             if (wi < nwords) {                               // warp-uniform
-                zpart += valid[x] ? ex2((unkey32(u[x]) - vmax) * c1) : 0.f;
                 const uint32_t dig = u[x] >> FSH;
                 const unsigned g = __ballot_sync(FULL, valid[x] && dig > b1);
                 const unsigned inb = __ballot_sync(FULL, valid[x] && dig == b1);
@@ -449,8 +437,9 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
             }
         }
     }
-    if (lane == 0) sc.redu[G::NW + warp] = wcount;           // second half of redu: free during group_sum
-    out.Z = group_sum<G>(zpart, sc.red, gtid);               // barriers also publish the bitmap and the lists
+    if (lane == 0) sc.redu[G::NW + warp] = wcount;
+    G::sync();                                               // publishes the bitmap and the lists
+    out.Z = Z_stream;
     out.need_tie = 0;
     POST_CLK(1);
     uint32_t m = 0;
@@ -462,40 +451,49 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
 
     // the threshold among the bin's m keys: `need` of them are wanted; remaining 22 bits as 8 + 8 + 6
     uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH, mask = ~0u << FSH, ceq = m;
+    // One 256-bin histogram per pass, all cleared up front, and every warp scanning the finished
+    // histogram for itself: one barrier per pass instead of three.
+    static_assert(CAND_MAX * 12 >= 3 * 256 * 4, "three histograms fit cand_val + cand_pos, free until the band step");
     uint32_t* h256 = reinterpret_cast<uint32_t*>(sc.cand_val);
     int shift = FSH;
+    if (ceq != need) {
+        for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
+        G::sync();
+    }
 #pragma unroll 1
     for (int pass = 0; pass < 3 && ceq != need; ++pass) {
         const int bits = pass < 2 ? 8 : 6;
         shift -= bits;
-        if (gtid < 256) h256[gtid] = 0;
-        G::sync();
+        uint32_t* hcur = h256 + pass * 256;
         for (uint32_t i = lane; i < my_n; i += 32) {
             const uint32_t u = seg_key[i];
-            if ((u & mask) == prefix) atomicAdd(&h256[(u >> shift) & ((1u << bits) - 1)], 1u);
+            if ((u & mask) == prefix) atomicAdd(&hcur[(u >> shift) & ((1u << bits) - 1)], 1u);
         }
         G::sync();
-        if (warp == 0) {                                     // 8 bins per lane, from the top
-            uint32_t c[8], sum = 0;
+        // 8 bins per lane, from the top; the lane whose range holds the need-th key knows the answer
+        uint32_t c[8], sum = 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) { c[i] = h256[255 - (lane * 8 + i)]; sum += c[i]; }
-            uint32_t incl = sum;
+        for (int i = 0; i < 8; ++i) { c[i] = hcur[255 - (lane * 8 + i)]; sum += c[i]; }
+        uint32_t incl = sum;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
-            uint32_t run = incl - sum;
-            if (run < need && need <= incl) {
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
+        uint32_t run = incl - sum, bin = 0, cnt = 0;
+        const bool mine = run < need && need <= incl;
+        if (mine) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (run + c[i] >= need) { sc.res[0] = 255 - (lane * 8 + i); sc.res[1] = run; sc.res[2] = c[i]; break; }
-                    run += c[i];
-                }
+            for (int i = 0; i < 8; ++i) {
+                if (run + c[i] >= need) { bin = 255 - (lane * 8 + i); cnt = c[i]; break; }
+                run += c[i];
             }
         }
-        G::sync();
-        prefix |= sc.res[0] << shift;
+        const int src = __ffs(__ballot_sync(FULL, mine)) - 1;    // exactly one lane
+        bin = __shfl_sync(FULL, bin, src);
+        run = __shfl_sync(FULL, run, src);
+        cnt = __shfl_sync(FULL, cnt, src);
+        prefix |= bin << shift;
         mask |= ((1u << bits) - 1) << shift;
-        need -= sc.res[1];
-        ceq = sc.res[2];
+        need -= run;
+        ceq = cnt;
     }
     POST_CLK(2);
     const uint32_t edge = prefix;                            // unprocessed low bits are zero

@@ -201,15 +201,22 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         const int t0 = c * CH + tid * 8;
         const int nvalid = min(8, n - t0);                   // positions of this thread's vector inside the sequence
+        __half2 mxc[4];                                      // |K| maximum of this chunk, kept only if the vector is inside
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mxc[e] = __float2half2_rn(0.f);
         for (int jb = 0; jb < r_pad; jb += RB, ++it) {
             ok = mbar_wait_bounded(&sh.full[s], parity, WAIT_LIMIT);
-            stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + tid, hm.qh + jb, r - jb, nvalid);
+            stage_fma<RB, CH / 8>(acc, mxc, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + tid, hm.qh + jb, r - jb);
             ok = __syncthreads_and(ok);                      // slot s fully consumed (or a wait gave up)
             if (!ok) break;
             if (warp == 0 && it + STAGES < total) issue(it + STAGES, s);
             if (++s == STAGES) { s = 0; parity ^= 1u; }
         }
         if (!ok) break;
+        if (nvalid > 0) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) mx[e] = __hmax2(mx[e], mxc[e]);
+        }
         uint32_t kk[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) kk[e] = key32(acc[e]);
@@ -284,20 +291,14 @@ sparq_split_scores_kernel(const sparq_half* __restrict__ q, const sparq_half* __
             float acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            if (nvalid > 0) {
-                uint32_t msk[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) msk[e] = (nvalid >= 2 * e + 2) ? 0xffffffffu : (nvalid == 2 * e + 1 ? 0x0000ffffu : 0u);
+            if (nvalid > 0) {                                // (the layout keeps zeros up to the end of the last vector)
                 for (int jb = 0; jb < r; jb += 8) {
                     uint4 v[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) v[u] = ld_stream(Kt_vec + (size_t)hm.i1[min(jb + u, r - 1)] * row_vecs + (t0 >> 3));
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
-                        if (jb + u < r) {
-                            v[u].x &= msk[0]; v[u].y &= msk[1]; v[u].z &= msk[2]; v[u].w &= msk[3];
-                            row_fma(acc, mx, v[u], hm.qh[jb + u]);
-                        }
+                        if (jb + u < r) row_fma(acc, mx, v[u], hm.qh[jb + u]);
                 }
 #pragma unroll
                 for (int e = 0; e < 8; ++e)

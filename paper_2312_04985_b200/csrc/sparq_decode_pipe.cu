@@ -61,6 +61,8 @@ struct PipeShared {
     uint64_t keys_full[NKB], keys_free[NKB];       // keys of a unit complete / post-processed
     uint32_t kmax[NKB];
     float kabs[NKB];
+    float zsum[NKB];                              // softmax denominator of the unit's approximate scores
+    float sred[2 * (SNT / 32)];
     float red[NPOST][2 * (GNT / 32)];
     uint32_t redu[NPOST][2 * (GNT / 32)];
     uint32_t res[NPOST][4];
@@ -263,6 +265,8 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
         if (hm.bh < 0 || sh.abort_flag) ++markers;           // forwarded to the post group below (group-uniform)
         if (hm.k_eff > 0) {
             uint32_t kmax = 0;
+            float zm = -CUDART_INF_F, zs = 0.f;              // this thread's running max (in log2 units) and sum of 2^(x - zm)
+            const float c1 = hm.inv_tau * LOG2E;
             __half2 mx[4];                                   // largest |K| among the valid streamed values
 #pragma unroll
             for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
@@ -274,6 +278,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 for (int e = 0; e < 8; ++e) acc[e] = 0.f;
                 const int t0 = c * CH + gtid * 8;
                 const int nvalid = min(8, n - t0);           // positions of this thread's vector inside the sequence
+                __half2 mxc[4];                              // |K| maximum of this chunk, kept only if the vector is inside
+#pragma unroll
+                for (int e = 0; e < 4; ++e) mxc[e] = __float2half2_rn(0.f);
                 for (int jb = 0; jb < r; jb += RB) {
 #ifdef SPARQ_PHASE_CLOCKS
                     const long long t_f0 = clock64();
@@ -282,8 +289,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 #ifdef SPARQ_PHASE_CLOCKS
                     ring_wait += clock64() - t_f0;
 #endif
-                    stage_fma<RB, CH / 8>(acc, mx, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid, hm.qh + jb, r - jb,
-                                          nvalid);
+                    stage_fma<RB, CH / 8>(acc, mxc, reinterpret_cast<const uint4*>(ring + s * STAGE_BYTES) + gtid, hm.qh + jb, r - jb);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sh.empty[s]);   // this warp is done with slot s
                     if (++s == STAGES) { s = 0; parity ^= 1u; }
@@ -291,6 +297,20 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                 uint32_t kk[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) kk[e] = key32(acc[e]);
+                if (nvalid > 0) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) mx[e] = __hmax2(mx[e], mxc[e]);
+                }
+                if (nvalid > 0) {                            // softmax statistics of this thread's keys (a3), online
+                    float cm = -CUDART_INF_F;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) if (e < nvalid) cm = fmaxf(cm, acc[e] * c1);
+                    const float nm = fmaxf(zm, cm);
+                    zs *= ex2(zm - nm);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) if (e < nvalid) zs += ex2(acc[e] * c1 - nm);
+                    zm = nm;
+                }
                 if (nvalid >= 8) {
                     *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
                     *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
@@ -304,7 +324,9 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
             }
             uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
             group_max2_u32<SG>(kmax, kabs_bits, sh.sredu, gtid);
-            if (gtid == 0) { sh.kmax[kb] = kmax; sh.kabs[kb] = __uint_as_float(kabs_bits); }
+            // Z = sum over threads of zs * 2^(zm - max), max = the largest logit in log2 units
+            const float Z = group_sum<SG>(zs > 0.f ? zs * ex2(zm - unkey32(kmax) * c1) : 0.f, sh.sred, gtid);
+            if (gtid == 0) { sh.kmax[kb] = kmax; sh.kabs[kb] = __uint_as_float(kabs_bits); sh.zsum[kb] = Z; }
         }
         SG::sync();                                          // every key of the unit is written
         if (gtid == 0) mbar_arrive(&sh.keys_full[kb]);
@@ -355,8 +377,8 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             sel.Z = 1.f; sel.need_tie = 0;
             if (false)
 #endif
-            if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, hist1_all + kb * FBINS, a.r, a.S_max,
-                                      Kt_head, sel))
+            if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sh.zsum[kb], sc, hist1_all + kb * FBINS, a.r,
+                                      a.S_max, Kt_head, sel))
                 sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
 #if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 2
             if (false)
