@@ -356,7 +356,7 @@ def run_b200(args):
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "us_per_step": 1e6 * e2e_s / e2e_steps, "api": "sparq_step_host (pinned host q, k_new, v_new -> host out)"},
-        "gpu_launches": 3 * args.steps,
+        "gpu_launches": 2 * args.steps,
         "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)

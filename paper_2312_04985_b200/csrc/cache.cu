@@ -6,32 +6,55 @@
 namespace sparq {
 namespace {
 
-// grid B*Hkv, D threads: thread c owns component c of the new token.
-__global__ void __launch_bounds__(D)
+// One CTA per sequence, one warp per KV head (warps stride over the heads when there are more than
+// 32 of them); lane l owns components 4l .. 4l+3 of the new token.  Every thread reads the old
+// length before the CTA-wide barrier and thread 0 stores the new one after it, so the whole append
+// is one launch.
+__global__ void __launch_bounds__(1024)
 cache_append_kernel(const sparq_half* __restrict__ k_new, const sparq_half* __restrict__ v_new,
                     sparq_half* __restrict__ K, sparq_half* __restrict__ Kt, sparq_half* __restrict__ V,
                     float* __restrict__ vsum, sparq_half* __restrict__ vbar,
-                    const int32_t* __restrict__ seq_lens, int Hkv, int S_max, int32_t* status) {
-    const int bh = blockIdx.x, c = threadIdx.x, b = bh / Hkv;
-    const int n = seq_lens[b];
-    if (n < 0 || n >= S_max) { if (c == 0) raise_status(status, SPARQ_DEV_CACHE_FULL); return; }
-    const uint16_t kc = k_new[(size_t)bh * D + c], vc = v_new[(size_t)bh * D + c];
-    const size_t head = (size_t)bh * S_max * D;
-    K[head + (size_t)n * D + c] = kc;
-    V[head + (size_t)n * D + c] = vc;
-    // the small non-contiguous write.  Invariant of the layout: the rest of the 16-byte vector that
-    // holds the last valid position is zero, so readers may take whole vectors without masking.
-    if ((n & 7) == 0) *reinterpret_cast<uint4*>(Kt + head + (size_t)c * S_max + n) = make_uint4(kc, 0u, 0u, 0u);
-    else Kt[head + (size_t)c * S_max + n] = kc;
-    float s = vsum[(size_t)bh * D + c] + __half2float(__ushort_as_half(vc));
-    vsum[(size_t)bh * D + c] = s;
-    vbar[(size_t)bh * D + c] = __half_as_ushort(__float2half_rn(s / (float)(n + 1)));
-}
-
-// runs after every head of every sequence has written at the old length
-__global__ void seq_bump_kernel(int32_t* seq_lens, int B, int S_max) {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B) { int n = seq_lens[b]; if (n >= 0 && n < S_max) seq_lens[b] = n + 1; }
+                    int32_t* __restrict__ seq_lens, int Hkv, int S_max, int32_t* status) {
+    static_assert(D == 128, "one warp covers a token: 32 lanes x 4 components");
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    const int c0 = lane * 4;
+    const int n = *reinterpret_cast<volatile const int32_t*>(seq_lens + b);
+    const bool ok = n >= 0 && n < S_max;
+    if (ok) {
+        for (int h = warp; h < Hkv; h += nw) {
+            const size_t bh = (size_t)b * Hkv + h, head = bh * S_max * D;
+            const uint2 kraw = *reinterpret_cast<const uint2*>(k_new + bh * D + c0);
+            const uint2 vraw = *reinterpret_cast<const uint2*>(v_new + bh * D + c0);
+            float4 s = *reinterpret_cast<const float4*>(vsum + bh * D + c0);
+            *reinterpret_cast<uint2*>(K + head + (size_t)n * D + c0) = kraw;
+            *reinterpret_cast<uint2*>(V + head + (size_t)n * D + c0) = vraw;
+            // the small non-contiguous writes.  Invariant of the layout: the rest of the 16-byte vector
+            // that holds the last valid position is zero, so readers may take whole vectors without masking.
+            const uint16_t kc[4] = {(uint16_t)(kraw.x & 0xffffu), (uint16_t)(kraw.x >> 16),
+                                    (uint16_t)(kraw.y & 0xffffu), (uint16_t)(kraw.y >> 16)};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                sparq_half* dst = Kt + head + (size_t)(c0 + u) * S_max + n;
+                if ((n & 7) == 0) *reinterpret_cast<uint4*>(dst) = make_uint4(kc[u], 0u, 0u, 0u);
+                else *dst = kc[u];
+            }
+            s.x += __half2float(__ushort_as_half((uint16_t)(vraw.x & 0xffffu)));
+            s.y += __half2float(__ushort_as_half((uint16_t)(vraw.x >> 16)));
+            s.z += __half2float(__ushort_as_half((uint16_t)(vraw.y & 0xffffu)));
+            s.w += __half2float(__ushort_as_half((uint16_t)(vraw.y >> 16)));
+            *reinterpret_cast<float4*>(vsum + bh * D + c0) = s;
+            const float inv = (float)(n + 1);
+            uint2 m;
+            m.x = (uint32_t)__half_as_ushort(__float2half_rn(s.x / inv)) | ((uint32_t)__half_as_ushort(__float2half_rn(s.y / inv)) << 16);
+            m.y = (uint32_t)__half_as_ushort(__float2half_rn(s.z / inv)) | ((uint32_t)__half_as_ushort(__float2half_rn(s.w / inv)) << 16);
+            *reinterpret_cast<uint2*>(vbar + bh * D + c0) = m;
+        }
+    }
+    __syncthreads();                                           // every thread has read the old length
+    if (threadIdx.x == 0) {
+        if (ok) seq_lens[b] = n + 1;
+        else raise_status(status, SPARQ_DEV_CACHE_FULL);
+    }
 }
 
 // grid (ceil(S_max/64), B*Hkv), 256 threads: Kt[:, t0:t0+64] = K[t0:t0+64, :]^T for t < n.
@@ -91,8 +114,8 @@ cudaError_t launch_cache_build(const sparq_half* K, const sparq_half* V, const i
 cudaError_t launch_cache_append(const sparq_half* k_new, const sparq_half* v_new, sparq_half* K, sparq_half* Kt,
                                 sparq_half* V, float* vsum, sparq_half* vbar, int32_t* seq_lens, int B, int Hkv,
                                 int S_max, int32_t* status, cudaStream_t st) {
-    cache_append_kernel<<<B * Hkv, D, 0, st>>>(k_new, v_new, K, Kt, V, vsum, vbar, seq_lens, Hkv, S_max, status);
-    seq_bump_kernel<<<(B + 255) / 256, 256, 0, st>>>(seq_lens, B, S_max);
+    const int threads = 32 * (Hkv < 32 ? Hkv : 32);
+    cache_append_kernel<<<B, threads, 0, st>>>(k_new, v_new, K, Kt, V, vsum, vbar, seq_lens, Hkv, S_max, status);
     return cudaGetLastError();
 }
 
