@@ -30,10 +30,14 @@ if ROOT not in sys.path:
 
 METRIC = "sparq_decode tokens*heads/s (us/step, HBM GB/s on compulsory bytes, speed-up vs dense_decode alongside)"
 UNIT = "tokens*heads/s"
-WORKLOAD = "c2"
+WORKLOAD = "c2"     # the workload the metric is quoted on; --workload runs the other configurations
 PERIOD = 64          # steps between rewinds of seq_lens (the cache would otherwise fill up)
 POOL = 16            # distinct (q, k_new, v_new) sets rotated through the steps
 L2_BYTES = 126e6
+# which decode plan the library picks per workload (kernels of the dominant launch; launches per step
+# = append kernel + decode kernels): long sequences and small batches take the two-kernel split plan
+DECODE_KERNEL = {"c1": "sparq_split_scores_kernel", "c3": "sparq_split_scores_kernel", "c4": "sparq_split_scores_kernel"}
+LAUNCHES_PER_STEP = {"c1": 3, "c2": 2, "c3": 3, "c4": 3}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
@@ -141,6 +145,11 @@ def time_oracle(case, n_units, reps=1):
     return len(seq), cores, times
 
 
+def _describe(name, case, B):
+    return "%s: B=%d Hq=%d Hkv=%d d=%d S_max=%d r=%d k=%d fp16 cache" % (name, B, case.Hq, case.Hkv, case.d, case.S_max,
+                                                                      case.r, case.k)
+
+
 def run_reference(args):
     """--impl reference: the oracle on the host cores, same metric and workload, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -148,24 +157,61 @@ def run_reference(args):
         return
     import torch
     from paper_2312_04985_b200 import synth
-    n_units = 64
+    spec = synth.SPECS[args.workload]
+    n_units = 64 if spec["S"] <= 4096 else 16
     dev = "cuda" if torch.cuda.is_available() else "cpu"
-    case = synth.make_case(WORKLOAD, device=dev, B=2)           # the sample only needs a few sequences' caches
+    case = synth.make_case(args.workload, device=dev, B=min(2, spec["B"]))   # the sample needs only a few sequences' caches
     from oracle import c_oracle
     c_oracle.build()
     U, cores, _ = time_oracle(case, n_units, reps=max(1, min(args.warmup, 1)))
     _, _, times = time_oracle(case, n_units, reps=max(1, min(args.steps, 5)))
     t = sum(times) / len(times)
     value = U / t
+    total_units = spec["B"] * spec["Hq"]
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": len(times), "warmup": 1, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "c2: B=64 Hq=Hkv=32 d=128 S=4096 r=32 k=128 fp16 cache",
-                       "sample": "%d of 2048 (batch, head) units per step" % U},
+            "config": {"workload": _describe(args.workload, case, spec["B"]),
+                       "sample": "%d of %d (batch, head) units per step" % (U, total_units)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": "%d (b,h) units of c2 per step, C float64 oracle, OpenMP over units" % U},
+                             "sample": "%d (b,h) units of %s per step, C float64 oracle, OpenMP over units"
+                                       % (U, args.workload)},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+class _Cache:
+    """One copy of the caches of a workload, at the state a period starts from."""
+
+    def __init__(self, torch, sparq, case, period, status):
+        dev = case.K.device
+        B, Hkv, d, S_max = case.B, case.Hkv, case.d, case.S_max
+        self.K, self.V = case.K.clone(), case.V.clone()
+        self.Kt = torch.zeros(B, Hkv, d, S_max, dtype=torch.float16, device=dev)
+        self.vsum = torch.zeros(B, Hkv, d, dtype=torch.float32, device=dev)
+        self.vbar = torch.zeros(B, Hkv, d, dtype=torch.float16, device=dev)
+        # a period of `period` appends ends at the length the workload names
+        self.seq_start = (case.seq_lens.to(torch.int32) + case.n_steps - period).clamp_(min=1)
+        self.seq_end = self.seq_start + period
+        self.seq_lens = self.seq_start.clone()
+        sparq.sparq_cache_build(self.K, self.V, self.seq_lens, self.Kt, self.vsum, self.vbar, status)
+        self.vsum_start = self.vsum.clone()
+        self.sparq, self.status = sparq, status
+
+    def rewind(self):
+        # lengths (and the running value sum) back to the start of a period; stream-ordered device
+        # copies of B and B*Hkv*d elements, inside the timed region
+        self.seq_lens.copy_(self.seq_start)
+        self.vsum.copy_(self.vsum_start)
+
+    def to_end(self):
+        self.seq_lens.copy_(self.seq_end)
+        self.sparq.sparq_cache_build(self.K, self.V, self.seq_lens, self.Kt, self.vsum, self.vbar, self.status)
+
+    def to_start(self):
+        self.seq_lens.copy_(self.seq_start)
+        self.sparq.sparq_cache_build(self.K, self.V, self.seq_lens, self.Kt, self.vsum, self.vbar, self.status)
+        self.vsum_start.copy_(self.vsum)
 
 
 def run_b200(args):
@@ -183,40 +229,31 @@ def run_b200(args):
     sparq.lib()                                                  # fail loudly if the library is missing
 
     # ---------------------------------------------------------------- workload (per rank, own seed)
-    case = synth.make_case(WORKLOAD, device=str(dev), seed=ranks.rank_seed(synth.SPECS[WORKLOAD]["seed"], rank),
-                           B=args.batch)
+    name = args.workload
+    case = synth.make_case(name, device=str(dev), seed=ranks.rank_seed(synth.SPECS[name]["seed"], rank), B=args.batch)
     B, Hq, Hkv, d, S_max, r, k = case.B, case.Hq, case.Hkv, case.d, case.S_max, case.r, case.k
     pool = synth.make_step_pool(case, POOL)
-    K, V = case.K, case.V
-    Kt = torch.zeros(B, Hkv, d, S_max, dtype=torch.float16, device=dev)
-    vsum = torch.zeros(B, Hkv, d, dtype=torch.float32, device=dev)
-    vbar = torch.zeros(B, Hkv, d, dtype=torch.float16, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    period = min(PERIOD, S_max - 8)
-    seq_start = torch.full((B,), S_max - period, dtype=torch.int32, device=dev)
-    seq_full = torch.full((B,), S_max, dtype=torch.int32, device=dev)
-    seq_lens = seq_start.clone()
-    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)    # state at the start of a period
-    vsum_start = vsum.clone()
+    period = min(case.n_steps if case.n_steps > 1 else PERIOD, S_max - 8)    # appends between rewinds of seq_lens
+    cache_bytes = 3 * case.K.numel() * 2
+    # caches smaller than a few L2 sizes are rotated over enough independent copies to defeat the L2
+    n_copies = 1 if cache_bytes > 4 * L2_BYTES else int(-(-4 * L2_BYTES // cache_bytes))
+    caches = [_Cache(torch, sparq, case, period, status) for _ in range(n_copies)]
+    del case.K, case.V
     out = torch.empty(B, Hq, d, dtype=torch.float16, device=dev)
     ws_bytes = sparq.sparq_workspace_bytes(B, Hq, Hkv, d, S_max, r, k)     # what the library says helps for these shapes
     dec_ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev) if ws_bytes else None
     torch.cuda.synchronize()
 
-    def rewind():
-        # start a period: lengths (and the running value sum) back to S - period; stream-ordered
-        # device copies of B and B*Hkv*d elements, inside the timed region
-        seq_lens.copy_(seq_start)
-        vsum.copy_(vsum_start)
-
     def step(i, ev=None):
-        if i % period == 0:
-            rewind()
+        c = caches[i % n_copies]
+        if (i // n_copies) % period == 0:
+            c.rewind()
         j = i % POOL
-        sparq.sparq_cache_append(pool["k_new"][j], pool["v_new"][j], K, Kt, V, vsum, vbar, seq_lens, status)
+        sparq.sparq_cache_append(pool["k_new"][j], pool["v_new"][j], c.K, c.Kt, c.V, c.vsum, c.vbar, c.seq_lens, status)
         if ev is not None:
             ev[0].record()
-        sparq.sparq_decode(pool["q"][j], K, Kt, V, vbar, seq_lens, r, k, out, workspace=dec_ws, status=status)
+        sparq.sparq_decode(pool["q"][j], c.K, c.Kt, c.V, c.vbar, c.seq_lens, r, k, out, workspace=dec_ws, status=status)
         if ev is not None:
             ev[1].record()
 
@@ -260,35 +297,40 @@ def run_b200(args):
     us_per_step = 1e3 * total_ms / args.steps
     units = B * Hq * world
     value = units / (us_per_step * 1e-6)
-    n_mean = sum(S_max - period + (i % period) + 1 for i in range(args.steps)) / args.steps
+    start_mean = float(caches[0].seq_start.float().mean().item())
+    n_mean = sum(start_mean + ((i // n_copies) % period) + 1 for i in range(args.steps)) / args.steps
     bytes_launch = B * Hq * compulsory_bytes_per_unit(n_mean, r, k, d)
     achieved = bytes_launch / (decode_us * 1e-6) / 1e9
     peak, peak_kind = _peaks()
 
-    # ---------------------------------------------------------------- dense_decode on the same cache
+    # ---------------------------------------------------------------- dense_decode on the same caches
     ws = torch.empty(max(sparq.dense_workspace_bytes(B, Hq, Hkv, d, S_max), 4), dtype=torch.uint8, device=dev)
-    seq_lens.copy_(seq_full)
-    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)    # whole cache valid: full-length comparison
+    for c in caches:
+        c.to_end()                                              # the lengths the workload names: full-length comparison
+    end_mean = float(caches[0].seq_end.float().mean().item())
     dn_steps = max(3, min(args.steps, 30))
-    for i in range(3):
-        sparq.dense_decode(pool["q"][i % POOL], K, V, seq_lens, out, workspace=ws, status=status)
-    barrier()
-    t_beg.record()
-    for i in range(dn_steps):
-        sparq.dense_decode(pool["q"][i % POOL], K, V, seq_lens, out, workspace=ws, status=status)
-    t_end.record()
-    barrier()
-    dense_us = max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / dn_steps)
-    # sparq_decode alone at the same full length, for the speed-up figure
-    for i in range(3):
-        sparq.sparq_decode(pool["q"][i % POOL], K, Kt, V, vbar, seq_lens, r, k, out, workspace=dec_ws, status=status)
-    barrier()
-    t_beg.record()
-    for i in range(dn_steps):
-        sparq.sparq_decode(pool["q"][i % POOL], K, Kt, V, vbar, seq_lens, r, k, out, workspace=dec_ws, status=status)
-    t_end.record()
-    barrier()
-    sparq_full_us = max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / dn_steps)
+
+    def dense(i):
+        c = caches[i % n_copies]
+        sparq.dense_decode(pool["q"][i % POOL], c.K, c.V, c.seq_lens, out, workspace=ws, status=status)
+
+    def sparse(i):
+        c = caches[i % n_copies]
+        sparq.sparq_decode(pool["q"][i % POOL], c.K, c.Kt, c.V, c.vbar, c.seq_lens, r, k, out, workspace=dec_ws, status=status)
+
+    def timed(fn):
+        for i in range(3):
+            fn(i)
+        barrier()
+        t_beg.record()
+        for i in range(dn_steps):
+            fn(i)
+        t_end.record()
+        barrier()
+        return max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / dn_steps)
+
+    dense_us = timed(dense)
+    sparq_full_us = timed(sparse)                                # sparq_decode alone at the same lengths, for the speed-up figure
 
     # ---------------------------------------------------------------- end to end from host buffers
     staging = torch.empty(sparq.sparq_step_host_staging_bytes(B, Hq, Hkv, d), dtype=torch.uint8, device=dev)
@@ -298,14 +340,14 @@ def run_b200(args):
     hout = torch.empty(B, Hq, d, dtype=torch.float16).pin_memory()
 
     def host_step(i):
-        if i % period == 0:
-            rewind()
+        c = caches[i % n_copies]
+        if (i // n_copies) % period == 0:
+            c.rewind()
         j = i % POOL
-        sparq.sparq_step_host(hq[j], hk[j], hv[j], K, Kt, V, vsum, vbar, seq_lens, r, k, hout, staging, status)
+        sparq.sparq_step_host(hq[j], hk[j], hv[j], c.K, c.Kt, c.V, c.vsum, c.vbar, c.seq_lens, r, k, hout, staging, status)
 
-    seq_lens.copy_(seq_start)
-    sparq.sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status)
-    vsum_start.copy_(vsum)
+    for c in caches:
+        c.to_start()
     for i in range(max(3, args.warmup // 2)):
         host_step(i)
     barrier()
@@ -318,6 +360,8 @@ def run_b200(args):
     e2e_value = units * e2e_steps / e2e_s
     h2d = (B * Hq * d + 2 * B * Hkv * d) * 2
     d2h = B * Hq * d * 2
+    if int(status.item()) != 0:
+        raise SystemExit("device status %s" % sparq.status_string(int(status.item())))
 
     if rank != 0:
         if world > 1:
@@ -329,34 +373,39 @@ def run_b200(args):
     if world == 1 and not args.no_cpu_baseline:
         from oracle import c_oracle
         c_oracle.build()
-        U, cores, times = time_oracle(case, 256, reps=1)        # warm-up (page-in, OpenMP pool) and calibration
+        case.K, case.V = caches[0].K, caches[0].V
+        n_sample = 256 if S_max <= 4096 else 32
+        U, cores, times = time_oracle(case, n_sample, reps=1)   # warm-up (page-in, OpenMP pool) and calibration
         reps = int(min(200, max(1, round(12.0 / max(times[0], 1e-3)))))             # about 12 s of CPU work
-        U, cores, times = time_oracle(case, 256, reps=reps)
+        U, cores, times = time_oracle(case, n_sample, reps=reps)
         cpu = {"value": U * reps / sum(times), "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "%d of %d (b,h) units of c2 (seeded sample), %d passes, C float64 oracle with OpenMP "
-                         "over units, %.1f s in all" % (U, B * Hq, reps, sum(times))}
+               "sample": "%d of %d (b,h) units of %s (seeded sample), %d passes, C float64 oracle with OpenMP "
+                         "over units, %.1f s in all" % (U, B * Hq, name, reps, sum(times))}
 
+    traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH if (name == "c2" and args.batch is None) else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 (fp16 cache; exact fp16 products summed in f32, threshold band re-decided in f64)",
         "data": "synthetic",
-        "config": {"workload": "c2: B=%d Hq=%d Hkv=%d d=%d S=%d r=%d k=%d fp16 cache, per GPU" % (B, Hq, Hkv, d, S_max, r, k),
-                   "step": "sparq_cache_append + sparq_decode; seq_lens rewound to S-%d every %d steps" % (period, period),
-                   "l2": "inputs larger than L2 (cache %.2f GB vs 126 MB L2); q/k/v rotate over %d sets"
-                         % (3 * K.numel() * 2 / 1e9, POOL),
+        "config": {"workload": _describe(name, case, B) + ", per GPU",
+                   "step": "sparq_cache_append + sparq_decode; mean length %.0f at the start of a period of %d steps, "
+                           "%.0f at its end, then seq_lens rewound" % (start_mean, period, end_mean),
+                   "l2": "%s (cache %.2f GB x %d cop%s vs 126 MB L2); q/k/v rotate over %d sets"
+                         % ("inputs larger than L2" if n_copies == 1 else "steps rotate over independent cache copies larger than L2 together",
+                            cache_bytes / 1e9, n_copies, "y" if n_copies == 1 else "ies", POOL),
                    "parallelism": "independent batches per GPU, no collective"},
         "us_per_step": us_per_step, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
         "dense_decode_us": dense_us, "speedup_vs_dense": dense_us / sparq_full_us,
-        "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, S_max, d) / (dense_us * 1e-6) / 1e9,
+        "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, end_mean, d) / (dense_us * 1e-6) / 1e9,
         "hbm_gbs_compulsory": achieved, "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "sparq_decode_pipe_kernel",
+                     "traffic": traffic, "kernel": DECODE_KERNEL.get(name, "sparq_decode_pipe_kernel"),
                      "algorithmic_bytes_per_launch": bytes_launch, "peak_kind": peak_kind + " (copy bandwidth)"},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "us_per_step": 1e6 * e2e_s / e2e_steps, "api": "sparq_step_host (pinned host q, k_new, v_new -> host out)"},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": LAUNCHES_PER_STEP.get(name, 2) * args.steps,
         "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
@@ -370,6 +419,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=["c1", "c2", "c3", "c4"],
+                    help="c2 is the configuration the metric is quoted on; the others are reported beside it")
     ap.add_argument("--batch", type=int, default=None, help="override B (profiling on a small case only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
