@@ -34,10 +34,10 @@ WORKLOAD = "c2"     # the workload the metric is quoted on; --workload runs the 
 PERIOD = 64          # steps between rewinds of seq_lens (the cache would otherwise fill up)
 POOL = 16            # distinct (q, k_new, v_new) sets rotated through the steps
 L2_BYTES = 126e6
-# which decode plan the library picks per workload (kernels of the dominant launch; launches per step
-# = append kernel + decode kernels): long sequences and small batches take the two-kernel split plan
-DECODE_KERNEL = {"c1": "sparq_split_scores_kernel", "c3": "sparq_split_scores_kernel", "c4": "sparq_split_scores_kernel"}
-LAUNCHES_PER_STEP = {"c1": 3, "c2": 2, "c3": 3, "c4": 3}
+# which decode kernel the library picks per workload (caches too long for the persistent kernel's
+# shared memory take the split-plan kernel); every step launches the append kernel and one decode kernel
+DECODE_KERNEL = {"c1": "sparq_decode_pipe_kernel", "c3": "sparq_split_kernel", "c4": "sparq_split_kernel"}
+LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
@@ -333,7 +333,7 @@ def run_b200(args):
     sparq_full_us = timed(sparse)                                # sparq_decode alone at the same lengths, for the speed-up figure
 
     # ---------------------------------------------------------------- end to end from host buffers
-    staging = torch.empty(sparq.sparq_step_host_staging_bytes(B, Hq, Hkv, d), dtype=torch.uint8, device=dev)
+    staging = torch.empty(sparq.sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k), dtype=torch.uint8, device=dev)
     hq = [pool["q"][j].cpu().pin_memory() for j in range(POOL)]
     hk = [pool["k_new"][j].cpu().pin_memory() for j in range(POOL)]
     hv = [pool["v_new"][j].cpu().pin_memory() for j in range(POOL)]

@@ -106,20 +106,24 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
  * sparq_decode -- the SparQ attention step (Section 4, Steps 1-3) for every (b, query head).
  * With n = seq_lens[b] and k_eff = min(k, n):
  *   i1 (r components, ties in |q| to the smaller index), tau (Eq. (9); an all-zero q uses tau = 1),
- *   l_hat[t] = sum_{j in i1} q_j K[t,j] / tau for t < n, accumulated in fp64 (Eq. (7)),
+ *   l_hat[t] = sum_{j in i1} q_j K[t,j] / tau for t < n (Eq. (7)): exact fp16 products summed in
+ *   fp32, with every position whose sum lies within the rounding-error bound of the selection
+ *   threshold re-decided by its fp64 sum, so that i2 is the set the fp64 definition selects,
  *   i2 = the k_eff largest l_hat (ties to the smaller position), alpha = sum_{t in i2} s_hat[t],
  *   y3 = softmax(q K[i2]^T / sqrt(d)) V[i2] in fp32 (Eq. (8)), out = alpha y3 + (1-alpha) vbar
  *   rounded to fp16 (Eq. (10)).  k == 0 gives out = vbar.
  * Optional outputs (each may be NULL): idx_r [B,Hq,r] int32 = i1 ascending; idx_k [B,Hq,k]
  * int32 = i2 ascending, unused tail -1; alpha [B,Hq] fp32.
  * workspace: optional device scratch; sparq_workspace_bytes() says how much helps for the given
- * shapes (0: none).  Three uses, results identical in all of them: fewer (batch, head) units
- * than SMs -- every sequence is cut into slices handled by different thread blocks (far lower
- * latency for batch-1 decode over a long cache); a cache too long for the persistent kernel -- the
- * scores take a streaming kernel of their own; more units than SMs on the persistent kernel -- 64
- * bytes for a counter from which the thread blocks draw their units, which evens out their
- * finishing times.  With workspace NULL or too small a plan without scratch is used.  The call
- * clears what it needs; contents are undefined afterwards.
+ * shapes (0: none).  Three uses, the selected sets identical in all of them (alpha and out may
+ * differ in their last bits, the softmax denominator being summed in another order): a cache too
+ * long for the persistent kernel's shared memory -- the approximate scores of a unit pass through
+ * the workspace (4 bytes per position); on top of that, fewer (batch, head) units than SMs with
+ * a lot to stream each -- every sequence is cut into slices handled by different thread blocks
+ * (far lower latency for batch-1 decode over a long cache); more units than SMs on the
+ * persistent kernel -- 64 bytes for a counter from which the thread blocks draw their units,
+ * which evens out their finishing times.  With workspace NULL or too small a plan without
+ * scratch is used.  The call clears what it needs; contents are undefined afterwards.
  */
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                  const sparq_half* vbar, const int32_t* seq_lens,
@@ -173,13 +177,15 @@ int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_ha
  * [B,Hq,d], k_new_host and v_new_host [B,Hkv,d] (fp16, ideally pinned) to the device, runs
  * sparq_cache_append then sparq_decode on `stream`, copies the result to out_host [B,Hq,d]
  * and waits for the stream.  The cache (K, Kt, V, vsum, vbar, seq_lens) stays resident on the
- * device.  staging: device scratch of at least sparq_step_host_staging_bytes() bytes.
+ * device.  staging: device scratch of at least sparq_step_host_staging_bytes() bytes (device
+ * copies of the four host tensors, then the workspace sparq_workspace_bytes() names for these
+ * shapes, at least 64 bytes).
  */
 int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, const sparq_half* v_new_host,
                     sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
                     int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
                     sparq_half* out_host, void* staging, size_t staging_bytes, int32_t* status, void* stream);
-size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d);
+size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k);
 
 #ifdef __cplusplus
 }

@@ -90,15 +90,24 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
                                   (cudaStream_t)stream));
 }
 
+// Which plan pays: the persistent kernel wherever one unit's keys fit its shared memory, except for
+// a few units (fewer than SMs) with a lot to stream each, which the split plan slices over all SMs.
+static bool split_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok) {
+    if (!pipe_ok) return true;
+    return units < n_sm && (size_t)2 * S_max * r > ((size_t)512 << 10);
+}
+
 size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
-    (void)r; (void)k;
+    (void)k;
     if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
-    // worth having: fewer units than SMs (slicing), or keys too long for the pipelined kernel
     const int n_sm = device_sm_count();
     const int splits = split_count(B * Hq, S_max, n_sm);
-    if (pipe_fits(S_max, device_smem_optin()) && (B * Hq >= n_sm || !splits))
-        return B * Hq > n_sm ? SPARQ_PIPE_WORKSPACE_BYTES : 0;   // the persistent kernel's unit counter
-    return splits ? split_scratch_bytes(B * Hq, S_max, splits) : 0;
+    const bool pipe_ok = pipe_fits(S_max, device_smem_optin());
+    const int plan = forced_plan();                          // a plan forced through the environment gets what it needs
+    if (splits && (plan == 3 || (plan == 0 && split_preferred(B * Hq, S_max, r, n_sm, pipe_ok))))
+        return split_scratch_bytes(B * Hq, S_max, splits);
+    if (pipe_ok) return B * Hq > n_sm ? SPARQ_PIPE_WORKSPACE_BYTES : 0;   // the persistent kernel's unit counter
+    return 0;
 }
 
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -115,7 +124,7 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     const int splits = split_count(B * Hq, S_max, n_sm);
     const bool ws_ok = splits && workspace && workspace_bytes >= split_scratch_bytes(B * Hq, S_max, splits);
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
-    const bool split_pays = B * Hq < n_sm || !pipe_fits(S_max, device_smem_optin());
+    const bool split_pays = split_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin()));
     if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
         return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
                                             alpha, status, splits, workspace, (cudaStream_t)stream));
@@ -159,9 +168,14 @@ int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_ha
     return rc(launch_dense_decode(q, K, V, seq_lens, B, Hq, Hkv, S_max, out, scratch, status, (cudaStream_t)stream));
 }
 
-size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d) {
-    if (B < 1 || Hq < 1 || Hkv < 1 || d < 1) return 0;
-    return ((size_t)2 * B * Hq * d + (size_t)2 * B * Hkv * d) * sizeof(sparq_half) + SPARQ_PIPE_WORKSPACE_BYTES;
+// device copies of q, out, k_new, v_new, then the workspace sparq_decode would like for these shapes
+static size_t step_host_ws_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
+    const size_t want = sparq_workspace_bytes(B, Hq, Hkv, d, S_max, r, k);
+    return want > SPARQ_PIPE_WORKSPACE_BYTES ? want : SPARQ_PIPE_WORKSPACE_BYTES;
+}
+size_t sparq_step_host_staging_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
+    if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
+    return ((size_t)2 * B * Hq * d + (size_t)2 * B * Hkv * d) * sizeof(sparq_half) + step_host_ws_bytes(B, Hq, Hkv, d, S_max, r, k);
 }
 
 int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, const sparq_half* v_new_host,
@@ -170,7 +184,7 @@ int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, cons
                     sparq_half* out_host, void* staging, size_t staging_bytes, int32_t* status, void* stream) {
     if (!q_host || !k_new_host || !v_new_host || !out_host) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
-    if (!staging || staging_bytes < sparq_step_host_staging_bytes(B, Hq, Hkv, d)) return SPARQ_ERR_WORKSPACE;
+    if (!staging || staging_bytes < sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k)) return SPARQ_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t nq = (size_t)B * Hq * d, nkv = (size_t)B * Hkv * d;
     sparq_half* q_dev = (sparq_half*)staging;
@@ -183,9 +197,9 @@ int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, cons
         return SPARQ_ERR_CUDA;
     int code = sparq_cache_append(k_dev, v_dev, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, d, S_max, status, stream);
     if (code != SPARQ_OK) return code;
-    void* ws = v_dev + nkv;                                  // the tail of the staging area: the decode's small workspace
+    void* ws = v_dev + nkv;                                  // the tail of the staging area: the decode's workspace
     code = sparq_decode(q_dev, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, out_dev, nullptr, nullptr, nullptr,
-                        ws, SPARQ_PIPE_WORKSPACE_BYTES, status, stream);
+                        ws, step_host_ws_bytes(B, Hq, Hkv, d, S_max, r, k), status, stream);
     if (code != SPARQ_OK) return code;
     if (cudaMemcpyAsync(out_host, out_dev, nq * sizeof(sparq_half), cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return SPARQ_ERR_CUDA;

@@ -219,6 +219,20 @@ __device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const Head
     }
     return acc;
 }
+// The same sum with 16 loads in flight at a time, for callers whose Kt reads come from far away
+// (long caches: every load a miss).  Not inlined: its registers stay out of the callers' hot loops.
+static __device__ __noinline__ double dot64_at_batched(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t) {
+    double acc = 0.0;
+    for (int j0 = 0; j0 < r; j0 += 16) {
+        uint16_t kv[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) kv[u] = j0 + u < r ? Kt_head[(size_t)hm.i1[j0 + u] * S_max + t] : (uint16_t)0;
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+            if (j0 + u < r) acc = fma(ldexp((double)hm.qf[hm.i1[j0 + u]], 1008), h2d_scalar(kv[u]), acc);
+    }
+    return acc;
+}
 
 // What a select variant hands to finish(): the selection bitmap sc.bm_sel (and, in the degenerate
 // path, the tie bitmap sc.bm_tie with need_tie of its lowest positions wanted) and the softmax
@@ -235,23 +249,35 @@ __device__ __forceinline__ float two_b(int r, float l1_sel, float kabs) {
 
 // Re-decide the positions listed in sc.cand_pos[0..n_cand) (all keys within 2B of the threshold) by
 // their fp64 sums of exact products: the need64 largest (ties to the lowest position) get their
-// bitmap bit set, the others cleared.  n_cand <= CAND_MAX <= group size.
-template <class G>
+// bitmap bit set, the others cleared.  n_cand <= CAND_MAX.
+template <class G, bool BATCHED = false>
 __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, const PostScratch& sc, uint32_t n_cand,
                                               uint32_t need64, const sparq_half* Kt_head, int S_max, int r) {
-    static_assert(CAND_MAX <= G::NT, "one thread per band candidate");
-    unsigned long long v = 0;
-    int t = 0;
-    if (gtid < n_cand) { t = sc.cand_pos[gtid]; v = key64(dot64_at(Kt_head, hm, S_max, r, t)); sc.cand_val[gtid] = v; }
-    G::sync();
-    if (gtid < n_cand) {
-        uint32_t rank = 0;
-        for (uint32_t i = 0; i < n_cand; ++i) {
-            const unsigned long long vi = sc.cand_val[i];
-            rank += (vi > v) || (vi == v && sc.cand_pos[i] < t);
+    constexpr int PER = (CAND_MAX + G::NT - 1) / G::NT;      // candidates per thread (1 for groups of 256)
+    unsigned long long v[PER];
+    int t[PER];
+#pragma unroll
+    for (int x = 0; x < PER; ++x) {
+        const uint32_t c = gtid + x * G::NT;
+        v[x] = 0; t[x] = 0;
+        if (c < n_cand) {
+            t[x] = sc.cand_pos[c];
+            v[x] = key64(BATCHED ? dot64_at_batched(Kt_head, hm, S_max, r, t[x]) : dot64_at(Kt_head, hm, S_max, r, t[x]));
+            sc.cand_val[c] = v[x];
         }
-        if (rank < need64) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
-        else atomicAnd(&sc.bm_sel[t >> 5], ~(1u << (t & 31)));
+    }
+    G::sync();
+#pragma unroll
+    for (int x = 0; x < PER; ++x) {
+        if (gtid + x * G::NT < n_cand) {
+            uint32_t rank = 0;
+            for (uint32_t i = 0; i < n_cand; ++i) {
+                const unsigned long long vi = sc.cand_val[i];
+                rank += (vi > v[x]) || (vi == v[x] && sc.cand_pos[i] < t[x]);
+            }
+            if (rank < need64) atomicOr(&sc.bm_sel[t[x] >> 5], 1u << (t[x] & 31));
+            else atomicAnd(&sc.bm_sel[t[x] >> 5], ~(1u << (t[x] & 31)));
+        }
     }
     G::sync();
 }
@@ -383,26 +409,28 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // Stages a4 + a3 when hist1 already holds the histogram of the keys' top FB bits.  One scan of the
 // keys builds the bitmap of everything above the threshold bin, the softmax denominator and the list
 // of the bin's own keys; the threshold is then resolved inside that short list, and the 2B band
-// around it re-decided in fp64 as in select_generic.  Clears hist1 for its next user.
+// around it re-decided in fp64 as in select_generic.  Clears hist1 for its next user (not with WIDE).
 // Returns false (for every thread of the group alike) when the short-cut does not apply -- a warp
 // meets more of the bin's keys than its list segment holds, or the band reaches outside the bin or holds too many keys -- and
 // the caller runs select_generic instead.
 // Z_stream: the softmax denominator relative to the largest key, accumulated by the stream stage.
-template <class G>
+template <class G, int FB_ = FB, bool WIDE = false>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
                                                  float kabs, float Z_stream, const PostScratch& sc, uint32_t* hist1, int r,
                                                  int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out) {
-    static_assert(G::NT >= 256, "thread i clears histogram word i");
+    constexpr int FSH_ = 32 - FB_, FBINS_ = 1 << FB_;         // first digit: the keys' top FB_ bits
+    static_assert(FSH_ > 16 && FSH_ <= 24, "the bin's remaining bits resolve as 8 + 8 + (FSH_ - 16)");
     const int lane = gtid & 31, warp = gtid >> 5;
     const int n = hm.n, k_eff = hm.k_eff;
     (void)kmax;
 
     POST_CLK_INIT();
     if (gtid < 4) sc.band[gtid] = 0;     // [0] band keys below the edge, [1] at/above it, [2] band list length
-    find_bin<G, FBINS>(hist1, (uint32_t)k_eff, sc.redu, sc.res, gtid);
+    find_bin<G, FBINS_>(hist1, (uint32_t)k_eff, sc.redu, sc.res, gtid);
     POST_CLK(0);
     const uint32_t b1 = sc.res[0], above = sc.res[1];
-    for (int i = gtid; i < FBINS / 4; i += G::NT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
+    if constexpr (!WIDE)                                     // (WIDE callers use a histogram once and may alias it with sc.hist)
+        for (int i = gtid; i < FBINS_ / 4; i += G::NT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
     // the bin's own keys: every warp appends to its own segment of the list (no atomics), in the
     // order it meets them
     constexpr int SEG = LIST_MAX / G::NW;                    // (key, position) pairs per warp
@@ -412,30 +440,76 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
 
     const int nwords = (n + 31) >> 5;
     uint32_t wcount = 0;                                     // this warp's list length (warp-uniform)
-    for (int w0 = warp; w0 < nwords; w0 += 4 * G::NW) {      // four words in flight per warp
-        uint32_t u[4];
-        bool valid[4];
+    if constexpr (WIDE) {
+        // Keys in global memory: one 16-byte vector per lane and load, four loads in flight, so that a
+        // warp has 2 KB on its way instead of 512 bytes.  A warp covers 128 positions (four bitmap
+        // words) per load: lane l holds positions 4l .. 4l+3 of the group, i.e. nibble l % 8 of
+        // bitmap word l / 8, and the eight lanes of a word OR their nibbles together.
+        const int ngroups = (n + 127) >> 7;
+        const unsigned oct = 0xffu << (lane & 24);           // the eight lanes that share a bitmap word
+        for (int g0 = warp; g0 < ngroups; g0 += 4 * G::NW) {
+            uint4 kv[4];
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
-            const int t = ((w0 + x * G::NW) << 5) + lane;
-            valid[x] = t < n;                                // also false for words past the end
-            u[x] = valid[x] ? keys[t] : 0u;
-        }
+            for (int x = 0; x < 4; ++x) {
+                const int t = ((g0 + x * G::NW) << 7) + lane * 4;
+                kv[x] = t < n ? *reinterpret_cast<const uint4*>(keys + t) : make_uint4(0u, 0u, 0u, 0u);
+            }
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {
-            const int wi = w0 + x * G::NW;
-            if (wi < nwords) {                               // warp-uniform
-                const uint32_t dig = u[x] >> FSH;
-                const unsigned g = __ballot_sync(FULL, valid[x] && dig > b1);
-                const unsigned inb = __ballot_sync(FULL, valid[x] && dig == b1);
-                if (lane == 0) sc.bm_sel[wi] = g;
-                if (inb) {
-                    const uint32_t slot = wcount + __popc(inb & lt);
-                    if ((inb >> lane & 1u) && slot < SEG) { seg_key[slot] = u[x]; seg_pos[slot] = (wi << 5) + lane; }
-                    wcount += __popc(inb);
+            for (int x = 0; x < 4; ++x) {
+                const int gi = g0 + x * G::NW;
+                if (gi < ngroups) {                          // warp-uniform
+                    const int t = (gi << 7) + lane * 4;
+                    const uint32_t u[4] = {kv[x].x, kv[x].y, kv[x].z, kv[x].w};
+                    uint32_t nib = 0, inb = 0;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const bool valid = t + e < n;
+                        const uint32_t dig = u[e] >> FSH_;
+                        nib |= (valid && dig > b1) ? 1u << e : 0u;
+                        inb |= (valid && dig == b1) ? 1u << e : 0u;
+                    }
+                    const uint32_t word = __reduce_or_sync(oct, nib << ((lane & 7) * 4));
+                    const int wi = (gi << 2) + (lane >> 3);
+                    if ((lane & 7) == 0 && wi < nwords) sc.bm_sel[wi] = word;
+                    if (__any_sync(FULL, inb != 0)) {        // the bin's own keys go to the warp's list
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const unsigned be = __ballot_sync(FULL, inb >> e & 1u);
+                            const uint32_t slot = wcount + __popc(be & lt);
+                            if ((inb >> e & 1u) && slot < SEG) { seg_key[slot] = u[e]; seg_pos[slot] = t + e; }
+                            wcount += __popc(be);
+                        }
+                    }
                 }
             }
         }
+    } else {
+        for (int w0 = warp; w0 < nwords; w0 += 4 * G::NW) {      // four words in flight per warp
+            uint32_t u[4];
+            bool valid[4];
+    #pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int t = ((w0 + x * G::NW) << 5) + lane;
+                valid[x] = t < n;                                // also false for words past the end
+                u[x] = valid[x] ? keys[t] : 0u;
+            }
+    #pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int wi = w0 + x * G::NW;
+                if (wi < nwords) {                               // warp-uniform
+                    const uint32_t dig = u[x] >> FSH_;
+                    const unsigned g = __ballot_sync(FULL, valid[x] && dig > b1);
+                    const unsigned inb = __ballot_sync(FULL, valid[x] && dig == b1);
+                    if (lane == 0) sc.bm_sel[wi] = g;
+                    if (inb) {
+                        const uint32_t slot = wcount + __popc(inb & lt);
+                        if ((inb >> lane & 1u) && slot < SEG) { seg_key[slot] = u[x]; seg_pos[slot] = (wi << 5) + lane; }
+                        wcount += __popc(inb);
+                    }
+                }
+            }
+        }
+
     }
     if (lane == 0) sc.redu[G::NW + warp] = wcount;
     G::sync();                                               // publishes the bitmap and the lists
@@ -449,20 +523,20 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     if (!fits) return false;
     const uint32_t my_n = min(wcount, (uint32_t)SEG);
 
-    // the threshold among the bin's m keys: `need` of them are wanted; remaining 22 bits as 8 + 8 + 6
-    uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH, mask = ~0u << FSH, ceq = m;
+    // the threshold among the bin's m keys: `need` of them are wanted; remaining bits as 8 + 8 + the rest
+    uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH_, mask = ~0u << FSH_, ceq = m;
     // One 256-bin histogram per pass, all cleared up front, and every warp scanning the finished
     // histogram for itself: one barrier per pass instead of three.
     static_assert(CAND_MAX * 12 >= 3 * 256 * 4, "three histograms fit cand_val + cand_pos, free until the band step");
     uint32_t* h256 = reinterpret_cast<uint32_t*>(sc.cand_val);
-    int shift = FSH;
+    int shift = FSH_;
     if (ceq != need) {
         for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
         G::sync();
     }
 #pragma unroll 1
     for (int pass = 0; pass < 3 && ceq != need; ++pass) {
-        const int bits = pass < 2 ? 8 : 6;
+        const int bits = pass < 2 ? 8 : FSH_ - 16;
         shift -= bits;
         uint32_t* hcur = h256 + pass * 256;
         for (uint32_t i = lane; i < my_n; i += 32) {
@@ -501,7 +575,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const float twoB = two_b(r, hm.l1_sel, kabs);
     const float edge_val = unkey32(edge);
     const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
-    if ((lo_key >> FSH) != b1 || (hi_key >> FSH) != b1) return false;   // keys outside the list may be in the band
+    if ((lo_key >> FSH_) != b1 || (hi_key >> FSH_) != b1) return false;   // keys outside the list may be in the band
 
     for (uint32_t i = lane; i < my_n; i += 32) {
         const uint32_t u = seg_key[i];
@@ -517,7 +591,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const uint32_t cnt_lo = sc.band[0], cnt_hi = sc.band[1], n_cand = sc.band[2];
     if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
         if (n_cand > CAND_MAX) return false;
-        redecide_band<G>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
+        redecide_band<G, WIDE>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
     }
     POST_CLK(3);
     return true;

@@ -17,7 +17,8 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
                                 int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                 int32_t* status, cudaStream_t stream);
 
-// split-S plan (sparq_decode.cu): two kernels and a scratch buffer, for fewer units than SMs
+// split-S plan (sparq_decode.cu): one CTA per (slice, unit) with the keys in a scratch buffer, for
+// caches too long for the persistent kernel and for few units with long sequences
 int split_count(int units, int S_max, int n_sm);
 size_t split_scratch_bytes(int units, int S_max, int splits);
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,

@@ -27,7 +27,6 @@ constexpr int BM_WORDS = 2048;           // bitmap capacity: 65536 positions
 using CTA = Group<NT, 0>;
 
 static_assert(post_scratch_bytes(CTA::NHW, BM_WORDS) <= RING_BYTES, "post-phase scratch must fit the dead ring");
-constexpr int SCRATCH_ONLY_BYTES = (int)((post_scratch_bytes(CTA::NHW, BM_WORDS) + 127) & ~(size_t)127);
 static_assert(RB <= 8, "HeadMeta::qh padding");
 
 
@@ -107,22 +106,16 @@ struct DecodeShared {
     uint32_t band[4];
 };
 
-// FROM_SCRATCH = false: the whole step.  FROM_SCRATCH = true: the second kernel of the split-S plan;
-// the keys of this unit were written to ws_keys by sparq_split_scores_kernel (with per-split maxima
-// in ws_part), so a2 is replaced by a copy of the keys into shared memory.
-template <bool FROM_SCRATCH>
 __global__ void __launch_bounds__(NT, 3)
 sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                     const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
                     const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
                     int Hq, int Hkv, int S_max, int r, int k,
                     sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
-                    float* __restrict__ alpha_out, int32_t* status,
-                    const uint32_t* __restrict__ ws_keys, const uint32_t* __restrict__ ws_part, int splits) {
+                    float* __restrict__ alpha_out, int32_t* status) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;                                       // a2: STAGES x [RB rows x CH positions] fp16
-    // [n] approximate-score keys, after the ring (or, without a2, after the post-phase scratch alone)
-    uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + (FROM_SCRATCH ? SCRATCH_ONLY_BYTES : RING_BYTES));
+    uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);  // [n] approximate-score keys
     __shared__ DecodeShared sh;
     HeadMeta& hm = sh.hm;
 
@@ -161,15 +154,6 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
 
     const sparq_half* Kt_head = Kt + kv_head * (size_t)D * S_max;
     uint32_t kmax = 0, kabs_bits = 0;
-    if constexpr (FROM_SCRATCH) {
-        // ---------------------------------------------------------------- a2 was done by the split kernel
-        const uint4* src = reinterpret_cast<const uint4*>(ws_keys + (size_t)bh * S_max);
-        for (int i = tid; i < (n + 3) / 4; i += NT) reinterpret_cast<uint4*>(keys)[i] = src[i];
-        for (int p = tid; p < splits; p += NT) {
-            kmax = max(kmax, ws_part[((size_t)bh * splits + p) * 2]);
-            kabs_bits = max(kabs_bits, ws_part[((size_t)bh * splits + p) * 2 + 1]);
-        }
-    } else {
     // ------------------------------------------------------------------ a2: stream r rows of Kt
     const int n8 = (n + 7) & ~7;                             // whole 16-byte vectors; n8 <= S_max
     const int n_chunks = (n8 + CH - 1) / CH;
@@ -238,7 +222,6 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     }
     PHASE_MARK(1);
     kabs_bits = __float_as_uint(mx_to_float(mx));
-    }
     group_max2_u32<CTA>(kmax, kabs_bits, sh.redu, tid);      // barriers: keys complete, ring is dead
 
     // ------------------------------------------------------------------ a3-a6 (scratch in the dead ring)
@@ -252,66 +235,198 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
 }
 
 // ---------------------------------------------------------------------------------- split-S plan
-// When there are fewer (batch, head) units than SMs (batch-1 decode over a long cache), one CTA
-// per unit leaves most of the GPU idle.  The split plan cuts every unit's sequence into `splits`
-// slices: grid (splits, units), 128 threads, each CTA repeats a1 (cheap) and streams its slice of
-// the r selected Kt rows with plain 128-bit loads (8 rows in flight per thread), writing the
-// slice's keys to a scratch buffer and its largest key / largest |K| beside them.  The second
-// kernel, sparq_decode_kernel<true>, one CTA per unit, picks the keys up and runs a3-a6 unchanged,
-// so the selected set is exactly the one of the unsplit plans.
-constexpr int SNT = 128;                 // threads of a scores CTA
-constexpr int SCH = SNT * 8;             // positions a scores CTA covers per pass
-using SCTA = Group<SNT, 0>;
+// For fewer (batch, head) units than SMs (batch-1 decode over a long cache) and for caches whose
+// keys do not fit the persistent kernel's shared memory: grid (splits, units), 128 threads, five
+// CTAs per SM.  Every unit's sequence is cut into `splits` interleaved slices; each CTA repeats
+// a1 (cheap) and streams its slice of the r selected Kt rows with plain 128-bit loads (16 rows in
+// flight per thread).  The keys go to a scratch buffer in global memory; the histogram of their top
+// SPLIT_FB bits, the largest key, the largest |K| and the softmax denominator stay in the CTA.
+//   splits == 1: the CTA goes straight on to a3-a6 with the keys it just wrote (they are read back
+//     out of the L2 while other CTAs of the SM stream: occupancy overlaps the two kinds of work).
+//   splits > 1: every CTA also leaves its histogram and statistics in the scratch buffer and takes a
+//     ticket from the unit's counter; the CTA that draws the last ticket sums the slices' histograms
+//     and runs a3-a6 for the unit.
+// The selection runs on the same keys with the same rules as in the other plans, so the selected
+// set is exactly theirs.
+constexpr int FNT = 128;                 // threads of a split-plan CTA
+constexpr int SCH = FNT * 8;             // positions a CTA covers per pass
+constexpr int SROWS = 16;                // Kt rows in flight per thread (16 with five CTAs per SM measured best)
+constexpr int SPLIT_CTAS = 5;            // resident CTAs per SM the kernel is compiled for
+constexpr int SPLIT_FB = 11;             // long sequences: a finer first digit keeps the threshold bin's list short
+constexpr int SPLIT_FBINS = 1 << SPLIT_FB;
+constexpr int PART_WORDS = 4;            // per (unit, slice): largest key, largest |K| bits, Z bits, unused
+using FCTA = Group<FNT, 0>;
 
-__global__ void __launch_bounds__(SNT)
-sparq_split_scores_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ Kt,
-                          const int32_t* __restrict__ seq_lens, int Hq, int Hkv, int S_max, int r, int k, int splits,
-                          uint32_t* __restrict__ ws_keys, uint32_t* __restrict__ ws_part, int32_t* __restrict__ idx_r) {
-    __shared__ HeadMeta hm;
-    __shared__ float red[2 * SCTA::NW];
-    __shared__ uint32_t redu[2 * SCTA::NW];
-    __shared__ uint32_t cnt[4];
+struct SplitShared {
+    HeadMeta hm;
+    int32_t i2[SPARQ_K_MAX];
+    float red[2 * FCTA::NW];
+    uint32_t redu[2 * FCTA::NW];
+    uint32_t res[4];
+    uint32_t band[4];
+    uint32_t cnt[4];
+    uint32_t ticket;
+};
+
+__global__ void __launch_bounds__(FNT, SPLIT_CTAS)
+sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
+                   const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
+                   const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
+                   int Hq, int Hkv, int S_max, int r, int k, int splits, int bm_words,
+                   sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
+                   float* __restrict__ alpha_out, int32_t* status,
+                   uint32_t* ws_keys, uint32_t* ws_part, uint32_t* ws_hist, unsigned int* ws_count) {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    // histogram of the keys' top bits; once the threshold bin is known the space becomes the select stage's list
+    uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn_smem);
+    static_assert(SPLIT_FBINS <= HIST_BINS, "the first-digit histogram aliases the select scratch's histogram");
+    __shared__ SplitShared sh;
+    HeadMeta& hm = sh.hm;
     const int tid = threadIdx.x, p = blockIdx.x, bh = blockIdx.y;
     const int b = bh / Hq, h = bh % Hq, hkv = h / (Hq / Hkv);
     const int n = seq_lens[b];
+    const size_t kv_head = (size_t)b * Hkv + hkv;
+    sparq_half* out_row = out + (size_t)bh * D;
+
+    if (n < 1 || n > S_max) {            // defined result, no trap (slice 0 writes it)
+        if (p == 0) {
+            if (tid == 0) { raise_status(status, SPARQ_DEV_BAD_SEQ_LEN); if (alpha_out) alpha_out[bh] = 0.f; }
+            if (tid < D) out_row[tid] = 0;
+            if (idx_r) for (int j = tid; j < r; j += FNT) idx_r[(size_t)bh * r + j] = -1;
+            if (idx_k) for (int j = tid; j < k; j += FNT) idx_k[(size_t)bh * k + j] = -1;
+        }
+        return;
+    }
+    const int k_eff = min(k, n);
+    PHASE_INIT();
+    for (int i = tid; i < SPLIT_FBINS / 4; i += FNT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) { hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; }
+    top_r_block<FCTA, 8>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.cnt);      // a1; its barriers also publish the cleared histogram
+    if (p == 0 && idx_r) for (int j = tid; j < r; j += FNT) idx_r[(size_t)bh * r + j] = hm.i1[j];
+    if (k_eff == 0) {                    // nothing to select: the output is the mean value vector
+        if (p == 0) {
+            if (tid < D) out_row[tid] = vbar[kv_head * D + tid];
+            if (tid == 0 && alpha_out) alpha_out[bh] = 0.f;
+        }
+        return;
+    }
+    PHASE_MARK(0);
+
+    // ------------------------------------------------------------------ a2 (+ a3 statistics) over this CTA's slice
+    const sparq_half* Kt_head = Kt + kv_head * (size_t)D * S_max;
+    uint32_t* keys = ws_keys + (size_t)bh * S_max;
+    const float c1 = hm.inv_tau * LOG2E;
     uint32_t kmax = 0;
+    float zm = -CUDART_INF_F, zs = 0.f;                      // running max (log2 units) and sum of 2^(x - zm)
     __half2 mx[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
-    if (n >= 1 && n <= S_max && k > 0) {                     // otherwise the second kernel reports / returns v_bar
-        top_r_block<SCTA, 8>(tid, q + (size_t)bh * D, r, hm, red, cnt);
-        if (p == 0 && idx_r) for (int j = tid; j < r; j += SNT) idx_r[(size_t)bh * r + j] = hm.i1[j];
-        const uint4* Kt_vec = reinterpret_cast<const uint4*>(Kt + ((size_t)b * Hkv + hkv) * (size_t)D * S_max);
+    {
+        const uint4* Kt_vec = reinterpret_cast<const uint4*>(Kt_head);
         const int row_vecs = S_max >> 3;
-        const int n_pass = ((n + 7) / 8 + SNT - 1) / SNT;    // passes of SCH positions over the whole sequence
-        uint32_t* keys = ws_keys + (size_t)bh * S_max;
+        const int n_pass = ((n + 7) / 8 + FNT - 1) / FNT;    // passes of SCH positions over the whole sequence
         for (int c = p; c < n_pass; c += splits) {           // this CTA's passes: c = p, p + splits, ...
             const int t0 = c * SCH + tid * 8;
             const int nvalid = min(8, n - t0);
+            if (nvalid <= 0) continue;                       // (the layout keeps zeros up to the end of the last vector)
             float acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-            if (nvalid > 0) {                                // (the layout keeps zeros up to the end of the last vector)
-                for (int jb = 0; jb < r; jb += 8) {
-                    uint4 v[8];
+            for (int jb = 0; jb < r; jb += SROWS) {
+                uint4 v[SROWS];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = ld_stream(Kt_vec + (size_t)hm.i1[min(jb + u, r - 1)] * row_vecs + (t0 >> 3));
+                for (int u = 0; u < SROWS; ++u) v[u] = ld_stream(Kt_vec + (size_t)hm.i1[min(jb + u, r - 1)] * row_vecs + (t0 >> 3));
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (jb + u < r) row_fma(acc, mx, v[u], hm.qh[jb + u]);
-                }
-#pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    if (e < nvalid) { const uint32_t kk = key32(acc[e]); keys[t0 + e] = kk; kmax = max(kmax, kk); }
+                for (int u = 0; u < SROWS; ++u)
+                    if (jb + u < r) row_fma(acc, mx, v[u], hm.qh[jb + u]);
             }
+            float cm = -CUDART_INF_F;                        // softmax statistics of these keys, online
+#pragma unroll
+            for (int e = 0; e < 8; ++e) if (e < nvalid) cm = fmaxf(cm, acc[e] * c1);
+            const float nm = fmaxf(zm, cm);
+            zs *= ex2(zm - nm);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) if (e < nvalid) zs += ex2(acc[e] * c1 - nm);
+            zm = nm;
+            uint32_t kk[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kk[e] = key32(acc[e]);
+            if (nvalid >= 8) {
+                *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+                *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                if (e < nvalid) {
+                    if (nvalid < 8) keys[t0 + e] = kk[e];
+                    kmax = max(kmax, kk[e]);
+                    atomicAdd(&hist1[kk[e] >> (32 - SPLIT_FB)], 1u);
+                }
         }
     }
-    else if (p == 0 && idx_r && (n < 1 || n > S_max)) {
-        for (int j = tid; j < r; j += SNT) idx_r[(size_t)bh * r + j] = -1;
-    }
     uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
-    group_max2_u32<SCTA>(kmax, kabs_bits, redu, tid);
-    if (tid == 0) { ws_part[((size_t)bh * splits + p) * 2] = kmax; ws_part[((size_t)bh * splits + p) * 2 + 1] = kabs_bits; }
+    group_max2_u32<FCTA>(kmax, kabs_bits, sh.redu, tid);     // barriers: the histogram and this CTA's keys are complete
+    // the slice's denominator relative to its own largest key
+    float Z = group_sum<FCTA>(zs > 0.f ? zs * ex2(zm - unkey32(kmax) * c1) : 0.f, sh.red, tid);
+    PHASE_MARK(1);
+
+    if (splits > 1) {
+        // leave this slice's results, take a ticket; only the last CTA of the unit goes on
+        const size_t slice0 = (size_t)bh * splits;
+        if (tid == 0)
+            *reinterpret_cast<uint4*>(ws_part + (slice0 + p) * PART_WORDS) = make_uint4(kmax, kabs_bits, __float_as_uint(Z), 0u);
+        uint4* hdst = reinterpret_cast<uint4*>(ws_hist + (slice0 + p) * SPLIT_FBINS);
+        for (int i = tid; i < SPLIT_FBINS / 4; i += FNT) hdst[i] = reinterpret_cast<const uint4*>(hist1)[i];
+        __threadfence();                                     // this thread's keys, histogram words, statistics: device-visible
+        __syncthreads();
+        if (tid == 0) sh.ticket = atomicAdd(&ws_count[bh], 1u);
+        __syncthreads();
+        if (sh.ticket != (uint32_t)(splits - 1)) return;
+        __threadfence();
+        // the unit's histogram: all slices summed (L2 reads: other SMs wrote them)
+        const uint4* hsrc = reinterpret_cast<const uint4*>(ws_hist + slice0 * SPLIT_FBINS);
+        for (int i = tid; i < SPLIT_FBINS / 4; i += FNT) {
+            uint4 s4 = __ldcg(hsrc + i);
+            for (int pp = 1; pp < splits; ++pp) {
+                const uint4 o = __ldcg(hsrc + (size_t)pp * (SPLIT_FBINS / 4) + i);
+                s4.x += o.x; s4.y += o.y; s4.z += o.z; s4.w += o.w;
+            }
+            reinterpret_cast<uint4*>(hist1)[i] = s4;
+        }
+        // largest key and |K| over the slices, then the denominators rescaled to the largest key
+        kmax = 0; kabs_bits = 0;
+        for (int pp = tid; pp < splits; pp += FNT) {
+            const uint4 part = __ldcg(reinterpret_cast<const uint4*>(ws_part + (slice0 + pp) * PART_WORDS));
+            kmax = max(kmax, part.x);
+            kabs_bits = max(kabs_bits, part.y);
+        }
+        group_max2_u32<FCTA>(kmax, kabs_bits, sh.redu, tid);
+        const float vmax = unkey32(kmax);
+        float zpart = 0.f;
+        for (int pp = tid; pp < splits; pp += FNT) {
+            const uint4 part = __ldcg(reinterpret_cast<const uint4*>(ws_part + (slice0 + pp) * PART_WORDS));
+            const float zp = __uint_as_float(part.z);
+            if (zp > 0.f) zpart += zp * ex2((unkey32(part.x) - vmax) * c1);
+        }
+        Z = group_sum<FCTA>(zpart, sh.red, tid);             // barriers: the summed histogram is complete as well
+    }
+
+    // ------------------------------------------------------------------ a3-a6 with the keys in global memory
+    PostScratch sc;
+    carve_post_scratch(sc, dyn_smem, FCTA::NHW, bm_words);
+    sc.i2 = sh.i2; sc.red = sh.red; sc.redu = sh.redu; sc.res = sh.res; sc.band = sh.band;
+    const float kabs = __uint_as_float(kabs_bits);
+    SelectResult sel;
+    if (!select_prefilled<FCTA, SPLIT_FB, true>(tid, hm, keys, kmax, kabs, Z, sc, hist1, r, S_max, Kt_head, sel)) {
+#ifdef SPARQ_PHASE_CLOCKS
+        if (tid == 0) atomicAdd(&g_phase_clocks[7], 1ull);
+#endif
+        sel = select_generic<FCTA>(tid, hm, keys, kmax, kabs, sc, r, S_max, Kt_head);
+    }
+    PHASE_MARK(2);
+    finish<FCTA, 4>(tid, hm, keys, kmax, sel, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
+                    vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
+    PHASE_MARK(3);
 }
 
 }  // namespace
@@ -325,9 +440,21 @@ extern "C" int sparq_debug_phase_clocks(unsigned long long* out16, int reset) {
 }
 #endif
 
+#ifdef SPARQ_PHASE_CLOCKS
+extern "C" int sparq_debug_post_clocks_split(unsigned long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    if (out16 && cudaMemcpyFromSymbol(out16, g_post_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_post_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+#endif
+
 size_t decode_static_smem() { return sizeof(DecodeShared); }
 size_t decode_dynamic_smem(int S_max) { return (size_t)RING_BYTES + (size_t)S_max * sizeof(uint32_t); }
-static size_t decode_dynamic_smem_from_scratch(int S_max) { return (size_t)SCRATCH_ONLY_BYTES + (size_t)S_max * sizeof(uint32_t); }
+static int post_bm_words(int S_max) { return (S_max + 127) / 128 * 4; }      // whole 16-byte groups of bitmap words
+static size_t post_dynamic_smem(int S_max) {
+    return (post_scratch_bytes(FCTA::NHW, post_bm_words(S_max)) + 127) & ~(size_t)127;
+}
 int decode_max_positions() { return BM_WORDS * 32; }
 
 cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -335,29 +462,27 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
                                 int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                 int32_t* status, cudaStream_t stream) {
     const size_t dyn = decode_dynamic_smem(S_max);
-    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
-    sparq_decode_kernel<false><<<B * Hq, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, idx_r,
-                                                            idx_k, alpha, status, nullptr, nullptr, 0);
+    sparq_decode_kernel<<<B * Hq, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, idx_r,
+                                                            idx_k, alpha, status);
     return cudaGetLastError();
 }
 
-// Slices per unit of the split plan: enough CTAs for about two per SM, at least one pass of SCH
-// positions per slice; 0 when the plan does not apply (a short cache).  With at least as many
-// units as SMs the answer is 1: no slicing, but still two kernels -- a pure streaming kernel at
-// high occupancy, then the latency-bound stages with the keys read back from the workspace --
-// which pays off when the keys of one unit fill most of an SM's shared memory.
+// Slices per unit of the split plan: enough CTAs for about two waves of resident CTAs, at least
+// one pass of SCH positions per slice; 0 when the plan does not apply (a short cache).
 int split_count(int units, int S_max, int n_sm) {
     if (n_sm <= 0 || S_max < 2 * SCH) return 0;
-    if (units >= n_sm) return 1;
-    const int want = (2 * n_sm + units - 1) / units;
+    const int want = (2 * SPLIT_CTAS * n_sm + units - 1) / units;      // about two waves of resident CTAs
     const int cap = (S_max + SCH - 1) / SCH;
     const int s = want < cap ? want : cap;
     return s < 1 ? 1 : s;
 }
 
 size_t split_scratch_bytes(int units, int S_max, int splits) {
-    return ((size_t)units * S_max + (size_t)units * splits * 2) * sizeof(uint32_t);
+    // keys; with slicing also per-slice statistics and histograms and the units' ticket counters
+    const size_t sliced = splits > 1 ? (size_t)units * splits * (PART_WORDS + SPLIT_FBINS) + (size_t)units : 0;
+    return ((size_t)units * S_max + sliced) * sizeof(uint32_t);
 }
 
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
@@ -367,13 +492,23 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
     const int units = B * Hq;
     uint32_t* ws_keys = static_cast<uint32_t*>(scratch);
     uint32_t* ws_part = ws_keys + (size_t)units * S_max;
-    const size_t dyn = decode_dynamic_smem_from_scratch(S_max);
-    cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    uint32_t* ws_hist = ws_part + (size_t)units * splits * PART_WORDS;
+    unsigned int* ws_count = ws_hist + (size_t)units * splits * SPLIT_FBINS;
+    const size_t dyn = post_dynamic_smem(S_max);
+    cudaError_t e = cudaFuncSetAttribute(sparq_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
-    sparq_split_scores_kernel<<<dim3(splits, units), SNT, 0, stream>>>(q, Kt, seq_lens, Hq, Hkv, S_max, r, k, splits,
-                                                                       ws_keys, ws_part, idx_r);
-    sparq_decode_kernel<true><<<units, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, nullptr,
-                                                          idx_k, alpha, status, ws_keys, ws_part, splits);
+    // Half of the SM's memory as shared memory holds the five CTAs; the other half stays L1, whose
+    // size bounds how many of the streaming loads can be in flight (measured: 50 % beats both 62 % and
+    // the driver's own choice).
+    e = cudaFuncSetAttribute(sparq_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
+    if (e != cudaSuccess) return e;
+    if (splits > 1) {
+        e = cudaMemsetAsync(ws_count, 0, (size_t)units * sizeof(unsigned int), stream);
+        if (e != cudaSuccess) return e;
+    }
+    sparq_split_kernel<<<dim3(splits, units), FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
+                                                                 post_bm_words(S_max), out, idx_r, idx_k, alpha, status,
+                                                                 ws_keys, ws_part, ws_hist, ws_count);
     return cudaGetLastError();
 }
 

@@ -69,7 +69,7 @@ def lib() -> ctypes.CDLL:
         L.sparq_step_host.restype = i
         L.sparq_step_host.argtypes = [vp] * 9 + [i] * 7 + [vp, vp, sz, vp, vp]
         L.sparq_step_host_staging_bytes.restype = sz
-        L.sparq_step_host_staging_bytes.argtypes = [i] * 4
+        L.sparq_step_host_staging_bytes.argtypes = [i] * 7
         _lib = L
     return _lib
 
@@ -109,8 +109,8 @@ def dense_workspace_bytes(B, Hq, Hkv, d, S_max) -> int:
     return int(lib().dense_workspace_bytes(B, Hq, Hkv, d, S_max))
 
 
-def sparq_step_host_staging_bytes(B, Hq, Hkv, d) -> int:
-    return int(lib().sparq_step_host_staging_bytes(B, Hq, Hkv, d))
+def sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k) -> int:
+    return int(lib().sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k))
 
 
 def sparq_cache_build(K, V, seq_lens, Kt, vsum, vbar, status=None):

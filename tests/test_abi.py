@@ -63,7 +63,7 @@ def test_host_visible_errors_need_no_device(lib):
     assert lib.dense_decode(one, one, one, one, 1, 32, 32, 128, 4096, one, n, 0, n, n) == sparq.ERR_WORKSPACE
     assert lib.dense_decode_static(one, one, one, one, 2, 1024, 32, 128, 4096, one, n, n) == sparq.ERR_STATIC_SCRATCH
     assert sparq.sparq_workspace_bytes(64, 32, 32, 128, 4096, 32, 128) == 0
-    assert sparq.sparq_step_host_staging_bytes(2, 4, 2, 128) == (2 * 2 * 4 * 128 + 2 * 2 * 2 * 128) * 2 + 64   # + decode workspace
+    assert sparq.sparq_step_host_staging_bytes(2, 4, 2, 128, 64, 4, 8) == (2 * 2 * 4 * 128 + 2 * 2 * 2 * 128) * 2 + 64   # + decode workspace
 
 
 def test_binding_refuses_cpu_tensors():
