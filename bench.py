@@ -41,7 +41,7 @@ LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 683.6e6   # 2 x (336.44 + 5.37) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 681.0e6   # 2 x (336.49 + 4.02) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md
 
 
 def compulsory_bytes_per_unit(n: float, r: int, k: int, d: int) -> float:

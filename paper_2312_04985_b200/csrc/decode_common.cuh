@@ -665,11 +665,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     float m = -CUDART_INF_F, l = 0.f, acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 1
-    for (int jb = 0; jb < 0; jb += G::NHW * RG) {
-#else
     for (int jb = 0; jb < k_eff; jb += G::NHW * RG) {        // trip count uniform across the group
-#endif
         uint4 kv[RG], vv[RG];
 #pragma unroll
         for (int u = 0; u < RG; ++u) {

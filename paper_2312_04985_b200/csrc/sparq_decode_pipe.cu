@@ -373,16 +373,9 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             const uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
             const sparq_half* Kt_head = a.Kt + kv_head * (size_t)D * a.S_max;
             SelectResult sel;
-#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 3
-            sel.Z = 1.f; sel.need_tie = 0;
-            if (false)
-#endif
             if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sh.zsum[kb], sc, hist1_all + kb * FBINS, a.r,
                                       a.S_max, Kt_head, sel))
                 sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
-#if defined(SPARQ_DBG_SKIP) && SPARQ_DBG_SKIP >= 2
-            if (false)
-#endif
             finish<PG, 4>(gtid, hm, keys, sh.kmax[kb], sel, sc, a.k, a.K + kv_head * (size_t)a.S_max * D,
                           a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
                           a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
