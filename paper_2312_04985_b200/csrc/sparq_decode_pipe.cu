@@ -150,12 +150,6 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
         const int k_eff = valid ? min(a.k, n) : 0;
         const uint16_t hb[4] = {(uint16_t)(qraw.x & 0xffffu), (uint16_t)(qraw.x >> 16), (uint16_t)(qraw.y & 0xffffu),
                                 (uint16_t)(qraw.y >> 16)};
-        // the next unit's query and length travel while this unit is ranked
-        const int bh_next = next_unit(a, bh, lane);
-        if (bh_next >= 0) {
-            qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh_next * D + lane * 4);
-            n_next = a.seq_lens[bh_next / a.Hq];
-        }
         wait_or_abort<200>(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
         CLK_BEGIN(t_a1);
         float qf[4], l1_all = 0.f;
@@ -204,7 +198,16 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.meta_full[m]);
         CLK_ADD(6, t_a1, lane == 0);
-        bh = bh_next;
+        // Only now draw the next unit and fetch its query and length: the stream group has a whole unit
+        // to work on meanwhile, and the first unit of the launch is not held up by the draw.  (Drawing
+        // later still -- once the stream group has started on this unit -- would leave fewer drawn but
+        // unstarted units per CTA at the end of the launch; it measured slower, the draw landing on the
+        // critical path.)
+        bh = next_unit(a, bh, lane);
+        if (bh >= 0) {
+            qraw = *reinterpret_cast<const uint2*>(a.q + (size_t)bh * D + lane * 4);
+            n_next = a.seq_lens[bh / a.Hq];
+        }
     }
 }
 
