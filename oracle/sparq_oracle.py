@@ -23,7 +23,8 @@ Readings taken where the paper is silent (each is listed in the design doc):
   * k is clipped to the sequence length; k = 0 returns v_bar;
   * an all-zero query gives tau := 1 (all approximate logits are 0);
   * under grouped-query attention every query head selects for itself over the KV head
-    ``h // g`` it shares.
+    ``h // g`` it shares (``sparq_decode``); the paper's own grouped variant, one selection
+    per KV head from sums over its query heads, is ``sparq_group_decode``.
 
 Pins (tests/test_oracle_*.py): Figure "SparQ for a single attention head" worked numbers,
 closed forms of Eq. (9), reduction to Eq. (2) at r = d_h and k = S, brute force over all
@@ -241,6 +242,118 @@ def dense_decode(q, K, V, seq_lens):
         for h in range(Hq):
             out[b, h] = dense_head(np.asarray(q[b, h], dtype=F64), K[b, h // g], V[b, h // g], n)
     return out
+
+
+# --------------------------------------------------------------------------- grouped queries
+# Section 4, "Grouped query attention": the g query heads that share a KV head select together.
+# Step 1 takes the top-r of |q| summed over the group; Step 2 takes the top-k of the approximate
+# scores summed over the group; temperature, scores, attention and alpha stay per query head.
+# Step 3 is applied per head, or left out (``realloc=False``: the paper dropped it for its
+# grouped-query models).  Readings: ties go to the smaller index in both selections; the Step 2
+# selection is on the summed softmax scores themselves (a sum over heads does not commute with the
+# softmax, so the logits cannot stand in for them here).
+def group_top_r(Q: np.ndarray, r: int):
+    """Step 1 for a group: Q [g, d_h]; the r largest components of sum_h |Q[h]|.
+    Returns (i1 ascending, relative gap at the boundary)."""
+    Q = np.asarray(Q, dtype=F64)
+    d = Q.shape[1]
+    if not 1 <= r <= d:
+        raise ValueError("r must be in [1, d_h]")
+    a = np.sum(np.abs(Q), axis=0)
+    order = _desc_order(a)
+    gap = math.inf if r == d else _rel_gap(a[order[r - 1]], a[order[r]])
+    return np.sort(order[:r]).astype(np.int64), gap
+
+
+def group_scores(Q: np.ndarray, K: np.ndarray, i1: np.ndarray, n: int):
+    """Eq. (7) for every head of the group over the shared component set i1: returns
+    (s_hat [g, n], tau [g]); tau is Eq. (9) per query head."""
+    Q = np.asarray(Q, dtype=F64)
+    g = Q.shape[0]
+    s_hat = np.zeros((g, n), dtype=F64)
+    tau = np.zeros(g, dtype=F64)
+    for h in range(g):
+        l_hat, tau[h] = approx_logits_fast(Q[h], K, i1, n)
+        s_hat[h] = softmax(l_hat)
+    return s_hat, tau
+
+
+def group_top_k(s_hat: np.ndarray, k: int):
+    """Step 2 for a group: the min(k, n) positions with the largest sum_h s_hat[h, t] (ties to the
+    smaller position), ascending; alpha [g] = each head's own score mass on that set (Step 3);
+    relative gap of the summed scores at the boundary."""
+    s_hat = np.asarray(s_hat, dtype=F64)
+    g, n = s_hat.shape
+    k_eff = max(0, min(int(k), n))
+    if k_eff == 0:
+        return np.zeros(0, dtype=np.int64), np.zeros(g, dtype=F64), math.inf
+    total = np.sum(s_hat, axis=0)
+    order = _desc_order(total)
+    sel = np.sort(order[:k_eff]).astype(np.int64)
+    alpha = np.sum(s_hat[:, sel], axis=1)
+    gap = math.inf if k_eff == n else _rel_gap(total[order[k_eff - 1]], total[order[k_eff]])
+    return sel, alpha, gap
+
+
+def group_from_i2(Q, K, V, v_bar, i2, alpha, realloc=True):
+    """Eq. (8) per head on the shared position set, then Eq. (10) per head (or not)."""
+    Q = np.asarray(Q, dtype=F64)
+    g, d = Q.shape
+    out = np.zeros((g, d), dtype=F64)
+    for h in range(g):
+        if len(i2) == 0:
+            out[h] = np.asarray(v_bar, dtype=F64)
+            continue
+        y = attend(Q[h], K, V, np.asarray(i2, dtype=np.int64))
+        out[h] = combine(float(alpha[h]), y, v_bar) if realloc else y
+    return out
+
+
+def group_from_i1(Q, K, V, v_bar, n, i1, k, realloc=True):
+    s_hat, tau = group_scores(Q, K, np.asarray(i1, dtype=np.int64), n)
+    i2, alpha, gap_k = group_top_k(s_hat, k)
+    out = group_from_i2(Q, K, V, v_bar, i2, alpha, realloc)
+    return dict(out=out, i2=i2, alpha=alpha, gap_k=gap_k, tau=tau, s_hat=s_hat)
+
+
+def sparq_group(Q, K, V, v_bar, n, r, k, realloc=True):
+    """The grouped step for one KV head: Q [g, d_h]; K, V [>= n, d_h]; v_bar [d_h]."""
+    if n < 1:
+        raise ValueError("sequence length must be >= 1")
+    i1, gap_r = group_top_r(Q, r)
+    res = group_from_i1(Q, K, V, v_bar, n, i1, k, realloc)
+    res.update(i1=i1, gap_r=gap_r)
+    return res
+
+
+def sparq_group_decode(q, K, V, seq_lens, r, k, v_bar=None, realloc=True):
+    """Grouped SparQ decode for q [B, Hq, d], K/V [B, Hkv, S_max, d], seq_lens [B]; query heads
+    hkv*g .. hkv*g + g - 1 form the group of KV head hkv.  Returns out [B,Hq,d], i1 [B,Hkv,r],
+    i2 [B,Hkv,k] (-1 padded), alpha [B,Hq], gap_r, gap_k [B,Hkv]."""
+    q = np.asarray(q)
+    B, Hq, d = q.shape
+    Hkv = K.shape[1]
+    g = Hq // Hkv
+    out = np.zeros((B, Hq, d), dtype=F64)
+    i1 = np.zeros((B, Hkv, r), dtype=np.int64)
+    i2 = -np.ones((B, Hkv, k), dtype=np.int64)
+    alpha = np.zeros((B, Hq), dtype=F64)
+    gap_r = np.zeros((B, Hkv), dtype=F64)
+    gap_k = np.zeros((B, Hkv), dtype=F64)
+    for b in range(B):
+        n = int(seq_lens[b])
+        for hkv in range(Hkv):
+            Kh = np.asarray(K[b, hkv, :n], dtype=F64)
+            Vh = np.asarray(V[b, hkv, :n], dtype=F64)
+            vb = mean_value(Vh, n) if v_bar is None else np.asarray(v_bar[b, hkv], dtype=F64)
+            res = sparq_group(np.asarray(q[b, hkv * g:(hkv + 1) * g], dtype=F64), Kh, Vh, vb, n, r, k, realloc)
+            out[b, hkv * g:(hkv + 1) * g] = res["out"]
+            i1[b, hkv] = res["i1"]
+            i2[b, hkv, : len(res["i2"])] = res["i2"]
+            alpha[b, hkv * g:(hkv + 1) * g] = res["alpha"]
+            gap_r[b, hkv] = res["gap_r"]
+            gap_k[b, hkv] = res["gap_k"]
+    return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k)
 
 
 # --------------------------------------------------------------------------- cache
