@@ -56,6 +56,7 @@ typedef uint16_t sparq_half;
 
 #define SPARQ_K_MAX 1024
 #define SPARQ_HEAD_DIM 128
+#define SPARQ_G_MAX 8           /* largest group (query heads per KV head) of sparq_decode_grouped */
 #define SPARQ_STATIC_SCRATCH_BYTES (8u << 20)   /* scratch built into the library for dense_decode_static */
 
 enum {
@@ -171,6 +172,30 @@ size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
  */
 int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
                         int B, int Hq, int Hkv, int d, int S_max, sparq_half* out, int32_t* status, void* stream);
+
+/*
+ * sparq_decode_grouped -- the grouped-query variant of the step (Section 4, "Grouped query
+ * attention"): the g = Hq / Hkv query heads of a KV head (heads hkv*g .. hkv*g + g - 1) select
+ * together.  i1 [B,Hkv,r] = the r components with the largest sum over the group of |q| (ties to
+ * the smaller index; the sums are exact); tau (Eq. (9)), l_hat and s_hat (Eq. (7)) per query
+ * head over that shared i1; i2 [B,Hkv,k] = the k_eff positions with the largest sum over the
+ * group of s_hat (equal sums to the smaller position); per head alpha = its own s_hat mass on
+ * i2, y3 = softmax(q K[i2]^T / sqrt(d)) V[i2] (Eq. (8)), and out = alpha y3 + (1 - alpha) vbar
+ * (Eq. (10)) when realloc != 0, out = y3 when realloc == 0 (the paper left Step 3 out for its
+ * grouped-query models).  The summed scores are evaluated in fp32 (about 1e-5 relative), so two
+ * positions whose sums differ by less than that may be selected the other way round than a
+ * float64 evaluation would.  g must be 1, 2, 4 or 8.  The r rows of Kt are streamed once per KV
+ * head instead of once per query head.
+ * workspace: required, sparq_grouped_workspace_bytes() bytes ((g + 1) * 4 bytes per position
+ * and KV head); contents undefined afterwards.  Optional outputs as in sparq_decode, with idx_r
+ * and idx_k per KV head.  Same error model as sparq_decode.
+ */
+int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                         const sparq_half* vbar, const int32_t* seq_lens,
+                         int B, int Hq, int Hkv, int d, int S_max, int r, int k, int realloc,
+                         sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
 
 /*
  * sparq_step_host -- one whole generation step driven from HOST buffers: copies q_host

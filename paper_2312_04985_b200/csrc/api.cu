@@ -141,6 +141,30 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
                                   status, (cudaStream_t)stream));
 }
 
+size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {
+    if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
+    return grouped_scratch_bytes(B, Hq, Hkv, S_max, grouped_slices(B * Hkv, S_max, device_sm_count()));
+}
+
+int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                         const sparq_half* vbar, const int32_t* seq_lens,
+                         int B, int Hq, int Hkv, int d, int S_max, int r, int k, int realloc,
+                         sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    const int g = Hq / Hkv;
+    if (g != 1 && g != 2 && g != 4 && g != 8) return SPARQ_ERR_BAD_SHAPE;
+    if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
+    if (grouped_dynamic_smem(S_max) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
+    const int slices = grouped_slices(B * Hkv, S_max, device_sm_count());
+    if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices) ||
+        reinterpret_cast<uintptr_t>(workspace) % 16 != 0)
+        return SPARQ_ERR_WORKSPACE;
+    return rc(launch_sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, realloc, out, idx_r, idx_k,
+                                          alpha, status, workspace, slices, (cudaStream_t)stream));
+}
+
 size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {
     if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
     return dense_scratch_bytes(B, Hq, Hkv, S_max);

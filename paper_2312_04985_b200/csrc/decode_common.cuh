@@ -250,7 +250,9 @@ __device__ __forceinline__ float two_b(int r, float l1_sel, float kabs) {
 // Re-decide the positions listed in sc.cand_pos[0..n_cand) (all keys within 2B of the threshold) by
 // their fp64 sums of exact products: the need64 largest (ties to the lowest position) get their
 // bitmap bit set, the others cleared.  n_cand <= CAND_MAX.
-template <class G, bool BATCHED = false>
+// BY_POS: the keys are final (no rounding-error band); the listed positions hold equal keys and the
+// lowest positions win.
+template <class G, bool BATCHED = false, bool BY_POS = false>
 __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, const PostScratch& sc, uint32_t n_cand,
                                               uint32_t need64, const sparq_half* Kt_head, int S_max, int r) {
     constexpr int PER = (CAND_MAX + G::NT - 1) / G::NT;      // candidates per thread (1 for groups of 256)
@@ -262,7 +264,8 @@ __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, cons
         v[x] = 0; t[x] = 0;
         if (c < n_cand) {
             t[x] = sc.cand_pos[c];
-            v[x] = key64(BATCHED ? dot64_at_batched(Kt_head, hm, S_max, r, t[x]) : dot64_at(Kt_head, hm, S_max, r, t[x]));
+            if constexpr (!BY_POS)
+                v[x] = key64(BATCHED ? dot64_at_batched(Kt_head, hm, S_max, r, t[x]) : dot64_at(Kt_head, hm, S_max, r, t[x]));
             sc.cand_val[c] = v[x];
         }
     }
@@ -284,7 +287,7 @@ __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, cons
 
 // Stages a4 + a3 from the keys alone (any n): MSB radix select over all keys, 11 + 11 + 10 bits,
 // then one pass for the softmax denominator, the bitmap and the threshold band.
-template <class G>
+template <class G, bool BY_POS = false>
 __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
                                                        float kabs, const PostScratch& sc, int r, int S_max,
                                                        const sparq_half* __restrict__ Kt_head) {
@@ -356,7 +359,18 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
         // sums of exact products; equal fp64 sums go to the lowest positions.
         const uint32_t need64 = cnt_hi - over;
         if (n_cand <= CAND_MAX) {
-            redecide_band<G>(gtid, hm, sc, n_cand, need64, Kt_head, S_max, r);
+            redecide_band<G, false, BY_POS>(gtid, hm, sc, n_cand, need64, Kt_head, S_max, r);
+        } else if constexpr (BY_POS) {
+            // many equal keys at the threshold: all of them tie, the first need64 positions are taken
+            need_tie = need64;
+            for (int wi = warp; wi < nwords; wi += G::NW) {
+                const int t = (wi << 5) + lane;
+                const uint32_t u = t < n ? keys[t] : 0u;
+                const unsigned g = __ballot_sync(FULL, t < n && u > hi_key);
+                const unsigned te = __ballot_sync(FULL, t < n && u >= lo_key && u <= hi_key);
+                if (lane == 0) { sc.bm_sel[wi] = g; sc.bm_tie[wi] = te; }
+            }
+            G::sync();
         } else {
             // many candidates (degenerate inputs, e.g. constant keys): radix select over their
             // 64-bit keys, 8 passes of 8 bits, then rebuild the bitmap
@@ -414,7 +428,7 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // meets more of the bin's keys than its list segment holds, or the band reaches outside the bin or holds too many keys -- and
 // the caller runs select_generic instead.
 // Z_stream: the softmax denominator relative to the largest key, accumulated by the stream stage.
-template <class G, int FB_ = FB, bool WIDE = false>
+template <class G, int FB_ = FB, bool WIDE = false, bool BY_POS = false>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
                                                  float kabs, float Z_stream, const PostScratch& sc, uint32_t* hist1, int r,
                                                  int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out) {
@@ -591,7 +605,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const uint32_t cnt_lo = sc.band[0], cnt_hi = sc.band[1], n_cand = sc.band[2];
     if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
         if (n_cand > CAND_MAX) return false;
-        redecide_band<G, WIDE>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
+        redecide_band<G, WIDE, BY_POS>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
     }
     POST_CLK(3);
     return true;
@@ -600,6 +614,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
 // Stages a5 and a6 for one unit from a finished selection: ascending index list from the bitmap(s),
 // alpha, gather of the selected K and V rows with online softmax, combine with v_bar.
 // RG: gathered K and V rows in flight per half-warp (register budget of the calling kernel).
+// realloc = false leaves Step 3 out (out = the restricted attention; alpha is still reported).
 // Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
 // group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
 template <class G, int RG>
@@ -607,9 +622,9 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
                                        const PostScratch& sc, int k, const sparq_half* __restrict__ K_head,
                                        const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
                                        sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
-                                       float* __restrict__ alpha_out) {
+                                       float* __restrict__ alpha_out, bool build_list = true, bool realloc = true) {
     const int n = hm.n, k_eff = hm.k_eff;
-    const int nwords = (n + 31) >> 5;
+    const int nwords = build_list ? (n + 31) >> 5 : 0;       // (a caller that kept sc.i2 from an earlier call skips the rebuild)
     const float vmax = unkey32(kmax);
     const float c1 = hm.inv_tau * LOG2E;
     const float Z = sel.Z;
@@ -732,7 +747,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
             L = fmaf(sc.merge[w * (D + 2) + D + 1], scl, L);
             s = fmaf(sc.merge[w * (D + 2) + gtid], scl, s);
         }
-        out_row[gtid] = __half_as_ushort(__float2half_rn(alpha * (s / L) + (1.f - alpha) * vb));
+        out_row[gtid] = __half_as_ushort(__float2half_rn(realloc ? alpha * (s / L) + (1.f - alpha) * vb : s / L));
     }
     if (gtid == 0 && alpha_out) *alpha_out = alpha;
     if (idx_k_row) for (int j = gtid; j < k; j += G::NT) idx_k_row[j] = (j < k_eff) ? sc.i2[j] : -1;
