@@ -56,6 +56,7 @@ typedef uint16_t sparq_half;
 
 #define SPARQ_K_MAX 1024
 #define SPARQ_HEAD_DIM 128
+#define SPARQ_S_MAX_WORKSPACE 262144   /* largest S_max of sparq_decode with a workspace, and of sparq_decode_grouped */
 #define SPARQ_G_MAX 8           /* largest group (query heads per KV head) of sparq_decode_grouped */
 #define SPARQ_STATIC_SCRATCH_BYTES (8u << 20)   /* scratch built into the library for dense_decode_static */
 
@@ -65,7 +66,8 @@ enum {
     SPARQ_ERR_BAD_SHAPE = 2,     /* B, Hq, Hkv, d or S_max outside the supported shapes          */
     SPARQ_ERR_BAD_RK = 3,        /* r or k out of range                                          */
     SPARQ_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than *_workspace_bytes()           */
-    SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds what the kernels' on-chip score buffer holds   */
+    SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds sparq_max_seq_len() (or, with a workspace,
+                                    SPARQ_S_MAX_WORKSPACE)                                      */
     SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
     SPARQ_ERR_STATIC_SCRATCH = 7,/* the problem needs more scratch than the library's fixed
                                     SPARQ_STATIC_SCRATCH_BYTES: use the call that takes a workspace */
@@ -78,7 +80,10 @@ enum {
 /* Human-readable name of a status code (static string, never NULL). */
 const char* sparq_status_string(int code);
 
-/* Largest S_max sparq_decode accepts on the current device (limited by shared memory). */
+/* Largest S_max sparq_decode accepts WITHOUT a workspace on the current device (the approximate
+ * scores of a unit then live in shared memory, 4 bytes per position).  With the workspace
+ * sparq_workspace_bytes() names, the scores go through it instead and the limit is
+ * SPARQ_S_MAX_WORKSPACE (only two bitmaps of S_max bits each stay in shared memory). */
 int sparq_max_seq_len(void);
 
 /*

@@ -101,7 +101,7 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     (void)k;
     if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
     const int n_sm = device_sm_count();
-    const int splits = split_count(B * Hq, S_max, n_sm);
+    const int splits = S_max <= SPARQ_S_MAX_WORKSPACE ? split_count(B * Hq, S_max, n_sm) : 0;
     const bool pipe_ok = pipe_fits(S_max, device_smem_optin());
     const int plan = forced_plan();                          // a plan forced through the environment gets what it needs
     if (splits && (plan == 3 || (plan == 0 && split_preferred(B * Hq, S_max, r, n_sm, pipe_ok))))
@@ -118,16 +118,19 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
-    if (S_max > sparq_max_seq_len()) return SPARQ_ERR_TOO_LONG;
     const int plan = forced_plan();
     const int n_sm = device_sm_count();
-    const int splits = split_count(B * Hq, S_max, n_sm);
+    const int splits = S_max <= SPARQ_S_MAX_WORKSPACE ? split_count(B * Hq, S_max, n_sm) : 0;
     const bool ws_ok = splits && workspace && workspace_bytes >= split_scratch_bytes(B * Hq, S_max, splits);
+    const bool too_long = S_max > sparq_max_seq_len();       // beyond shared memory only the split plan's scratch buffer helps
+    if (too_long && !ws_ok)
+        return S_max <= SPARQ_S_MAX_WORKSPACE && (plan == 0 || plan == 3) ? SPARQ_ERR_WORKSPACE : SPARQ_ERR_TOO_LONG;
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
     const bool split_pays = split_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin()));
     if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
         return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
                                             alpha, status, splits, workspace, (cudaStream_t)stream));
+    if (too_long) return SPARQ_ERR_TOO_LONG;                 // a plan without scratch was forced
     const bool fits = pipe_fits(S_max, device_smem_optin());
     if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
     if (fits && plan != 1) {
@@ -156,7 +159,7 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
     const int g = Hq / Hkv;
     if (g != 1 && g != 2 && g != 4 && g != 8) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
-    if (grouped_dynamic_smem(S_max) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
+    if (S_max > SPARQ_S_MAX_WORKSPACE || grouped_dynamic_smem(S_max) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
     const int slices = grouped_slices(B * Hkv, S_max, device_sm_count());
     if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices) ||
         reinterpret_cast<uintptr_t>(workspace) % 16 != 0)

@@ -110,6 +110,25 @@ def test_split_plan_unsliced_many_units():
     assert total == 1536 and waived <= 5
 
 
+def test_cache_longer_than_shared_memory_goes_through_the_workspace():
+    """S_max beyond sparq_max_seq_len(): refused without a workspace, exact with one."""
+    S = 65536
+    assert S > sparq.sparq_max_seq_len()
+    c = synth.make_case("c3", device="cuda", B=1, Hq=2, Hkv=2, S=S, ragged=(50000, 65000))
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    waived, total = H.run_case_all_heads(c, "long cache")
+    assert total == 2 and waived == 0
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
+    q = c.q_steps[0].cuda()
+    with pytest.raises(sparq.SparqError) as e:
+        sparq.sparq_decode(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, c.r, c.k, torch.empty_like(q))
+    assert e.value.code == sparq.ERR_WORKSPACE
+    with H.decode_plan("simple"), pytest.raises(sparq.SparqError) as e:
+        sparq.sparq_decode(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, c.r, c.k, torch.empty_like(q))
+    assert e.value.code == sparq.ERR_TOO_LONG
+
+
 def test_dense_decode_on_workloads():
     for name, kw in (("c1", {}), ("c3", dict(B=2, S=5000, backend="numpy")),
                      ("c4", dict(B=3, n_steps=1, ragged=(700, 2500), backend="numpy"))):
