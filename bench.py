@@ -331,6 +331,18 @@ def run_b200(args):
 
     dense_us = timed(dense)
     sparq_full_us = timed(sparse)                                # sparq_decode alone at the same lengths, for the speed-up figure
+    # the variant that stores K once: stage a2 reads whole rows of K (d/r times the bytes of the Kt stream)
+    ws1 = torch.empty(sparq.sparq_1xk_workspace_bytes(B, Hq, Hkv, d, S_max), dtype=torch.uint8, device=dev)
+
+    def one_k_fn(i):
+        c = caches[i % n_copies]
+        sparq.sparq_decode_1xk(pool["q"][i % POOL], c.K, c.V, c.vbar, c.seq_lens, r, k, out, ws1, status=status)
+
+    k1_us = timed(one_k_fn)
+    del ws1
+    k1_bytes = B * Hq * (2.0 * end_mean * d + 4.0 * k * d + 6.0 * d)      # whole K rows per query head: sector granularity
+    one_k = {"us": k1_us, "bytes_at_sector_granularity": k1_bytes, "hbm_gbs": k1_bytes / (k1_us * 1e-6) / 1e9,
+             "speedup_vs_dense": dense_us / k1_us, "slowdown_vs_two_copies": k1_us / sparq_full_us}
     grouped = None
     if Hq != Hkv:
         # the paper's grouped-query variant (one selection per KV head) on the same caches, beside the per-head path
@@ -410,6 +422,7 @@ def run_b200(args):
                    "parallelism": "independent batches per GPU, no collective"},
         "us_per_step": us_per_step, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
         "dense_decode_us": dense_us, "speedup_vs_dense": dense_us / sparq_full_us, "sparq_decode_grouped": grouped,
+        "sparq_decode_1xk": one_k,
         "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, end_mean, d) / (dense_us * 1e-6) / 1e9,
         "hbm_gbs_compulsory": achieved, "frac_of_8tbs": achieved / 8000.0,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -203,6 +203,20 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
 size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
 
 /*
+ * sparq_decode_1xk -- sparq_decode for a cache that stores K once (no transposed copy Kt): the
+ * variant the paper measures beside the K-stored-twice one (Section 6.1) and leaves open because
+ * of the 50 % extra memory Kt costs.  Stage a2 reads whole rows of K (the r selected components
+ * of a row are spread over all its 32-byte sectors, so the step moves d/r times the bytes of the
+ * Kt stream); results are those of sparq_decode (same selected sets; alpha and out to the last
+ * bits).  workspace: required, sparq_1xk_workspace_bytes() bytes; contents undefined afterwards.
+ */
+int sparq_decode_1xk(const sparq_half* q, const sparq_half* K, const sparq_half* V, const sparq_half* vbar,
+                     const int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                     sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                     void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+size_t sparq_1xk_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
+
+/*
  * sparq_step_host -- one whole generation step driven from HOST buffers: copies q_host
  * [B,Hq,d], k_new_host and v_new_host [B,Hkv,d] (fp16, ideally pinned) to the device, runs
  * sparq_cache_append then sparq_decode on `stream`, copies the result to out_host [B,Hq,d]

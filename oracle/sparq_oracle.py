@@ -16,7 +16,7 @@ Notation follows the paper: ``q`` query (d_h components), ``K``/``V`` key/value 
 sequence positions, ``s_hat`` approximate scores, ``tau`` the softmax temperature,
 ``alpha`` the approximate score mass of the top-k set, ``v_bar`` the running mean of V.
 
-Readings taken where the paper is silent (each is listed in the design doc):
+Readings taken where the paper is silent:
   * ties in either top-k resolve to the smaller index;
   * the top-k is taken over the approximate logits (softmax is strictly increasing, so
     this is the top-k of s_hat whenever s_hat does not underflow);

@@ -129,7 +129,7 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     const bool split_pays = split_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin()));
     if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
         return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
-                                            alpha, status, splits, workspace, (cudaStream_t)stream));
+                                            alpha, status, splits, workspace, false, (cudaStream_t)stream));
     if (too_long) return SPARQ_ERR_TOO_LONG;                 // a plan without scratch was forced
     const bool fits = pipe_fits(S_max, device_smem_optin());
     if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
@@ -142,6 +142,32 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     }
     return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
                                   status, (cudaStream_t)stream));
+}
+
+static int one_k_splits(int units, int S_max) {
+    const int s = split_count(units, S_max, device_sm_count());
+    return s < 1 ? 1 : s;
+}
+
+size_t sparq_1xk_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {
+    if (bad_common(B, Hq, Hkv, d, S_max)) return 0;
+    return split_scratch_bytes(B * Hq, S_max, one_k_splits(B * Hq, S_max));
+}
+
+int sparq_decode_1xk(const sparq_half* q, const sparq_half* K, const sparq_half* V, const sparq_half* vbar,
+                     const int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                     sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                     void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (!q || !K || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
+    if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
+    if (S_max > SPARQ_S_MAX_WORKSPACE) return SPARQ_ERR_TOO_LONG;
+    const int splits = one_k_splits(B * Hq, S_max);
+    if (!workspace || workspace_bytes < split_scratch_bytes(B * Hq, S_max, splits) ||
+        reinterpret_cast<uintptr_t>(workspace) % 16 != 0)
+        return SPARQ_ERR_WORKSPACE;
+    return rc(launch_sparq_decode_split(q, K, nullptr, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
+                                        status, splits, workspace, true, (cudaStream_t)stream));
 }
 
 size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {

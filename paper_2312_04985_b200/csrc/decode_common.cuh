@@ -211,22 +211,27 @@ __device__ __forceinline__ void zero_hist(uint32_t* hist, int gtid) {
 
 // fp64 sum of the exact products of the selected query components with position t of the r
 // selected Kt rows, in i1 order: bit for bit the float64 oracle's accumulation.
-__device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t) {
+// Element (component c, position t) is Kt_head[c * S_max + t * t_stride]: the transposed cache with t_stride = 1, or
+// the row-major K with S_max := 1 and t_stride := d_h (the variant that stores K once).
+__device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t,
+                                           int t_stride = 1) {
     double acc = 0.0;
     for (int j = 0; j < r; ++j) {
         const int c = hm.i1[j];
-        acc = fma(ldexp((double)hm.qf[c], 1008), h2d_scalar(Kt_head[(size_t)c * S_max + t]), acc);
+        acc = fma(ldexp((double)hm.qf[c], 1008), h2d_scalar(Kt_head[(size_t)c * S_max + (size_t)t * t_stride]), acc);
     }
     return acc;
 }
 // The same sum with 16 loads in flight at a time, for callers whose Kt reads come from far away
 // (long caches: every load a miss).  Not inlined: its registers stay out of the callers' hot loops.
-static __device__ __noinline__ double dot64_at_batched(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t) {
+static __device__ __noinline__ double dot64_at_batched(const sparq_half* Kt_head, const HeadMeta& hm, int S_max, int r, int t,
+                                                       int t_stride = 1) {
     double acc = 0.0;
     for (int j0 = 0; j0 < r; j0 += 16) {
         uint16_t kv[16];
 #pragma unroll
-        for (int u = 0; u < 16; ++u) kv[u] = j0 + u < r ? Kt_head[(size_t)hm.i1[j0 + u] * S_max + t] : (uint16_t)0;
+        for (int u = 0; u < 16; ++u)
+            kv[u] = j0 + u < r ? Kt_head[(size_t)hm.i1[j0 + u] * S_max + (size_t)t * t_stride] : (uint16_t)0;
 #pragma unroll
         for (int u = 0; u < 16; ++u)
             if (j0 + u < r) acc = fma(ldexp((double)hm.qf[hm.i1[j0 + u]], 1008), h2d_scalar(kv[u]), acc);
@@ -254,7 +259,8 @@ __device__ __forceinline__ float two_b(int r, float l1_sel, float kabs) {
 // lowest positions win.
 template <class G, bool BATCHED = false, bool BY_POS = false>
 __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, const PostScratch& sc, uint32_t n_cand,
-                                              uint32_t need64, const sparq_half* Kt_head, int S_max, int r) {
+                                              uint32_t need64, const sparq_half* Kt_head, int S_max, int r,
+                                              int t_stride = 1) {
     constexpr int PER = (CAND_MAX + G::NT - 1) / G::NT;      // candidates per thread (1 for groups of 256)
     unsigned long long v[PER];
     int t[PER];
@@ -265,7 +271,8 @@ __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, cons
         if (c < n_cand) {
             t[x] = sc.cand_pos[c];
             if constexpr (!BY_POS)
-                v[x] = key64(BATCHED ? dot64_at_batched(Kt_head, hm, S_max, r, t[x]) : dot64_at(Kt_head, hm, S_max, r, t[x]));
+                v[x] = key64(BATCHED ? dot64_at_batched(Kt_head, hm, S_max, r, t[x], t_stride)
+                                     : dot64_at(Kt_head, hm, S_max, r, t[x], t_stride));
             sc.cand_val[c] = v[x];
         }
     }
@@ -290,7 +297,7 @@ __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, cons
 template <class G, bool BY_POS = false>
 __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
                                                        float kabs, const PostScratch& sc, int r, int S_max,
-                                                       const sparq_half* __restrict__ Kt_head) {
+                                                       const sparq_half* __restrict__ Kt_head, int t_stride = 1) {
     const int lane = gtid & 31, warp = gtid >> 5;
     const int n = hm.n, k_eff = hm.k_eff;
     const float inv_tau = hm.inv_tau;
@@ -359,7 +366,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
         // sums of exact products; equal fp64 sums go to the lowest positions.
         const uint32_t need64 = cnt_hi - over;
         if (n_cand <= CAND_MAX) {
-            redecide_band<G, false, BY_POS>(gtid, hm, sc, n_cand, need64, Kt_head, S_max, r);
+            redecide_band<G, false, BY_POS>(gtid, hm, sc, n_cand, need64, Kt_head, S_max, r, t_stride);
         } else if constexpr (BY_POS) {
             // many equal keys at the threshold: all of them tie, the first need64 positions are taken
             need_tie = need64;
@@ -383,7 +390,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
                 for (int t = gtid; t < n; t += G::NT) {
                     const uint32_t u = keys[t];
                     if (u >= lo_key && u <= hi_key) {
-                        const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t));
+                        const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t, t_stride));
                         if ((v & m64) == p64) atomicAdd(&sc.hist[(uint32_t)(v >> shift) & 255u], 1u);
                     }
                 }
@@ -399,7 +406,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
                 const uint32_t u = t < n ? keys[t] : 0u;
                 bool s_ = t < n && u > hi_key, tie = false;
                 if (t < n && u >= lo_key && u <= hi_key) {
-                    const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t));
+                    const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t, t_stride));
                     s_ = v > p64;
                     tie = v == p64;
                 }
@@ -431,7 +438,8 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 template <class G, int FB_ = FB, bool WIDE = false, bool BY_POS = false>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
                                                  float kabs, float Z_stream, const PostScratch& sc, uint32_t* hist1, int r,
-                                                 int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out) {
+                                                 int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out,
+                                                 int t_stride = 1) {
     constexpr int FSH_ = 32 - FB_, FBINS_ = 1 << FB_;         // first digit: the keys' top FB_ bits
     static_assert(FSH_ > 16 && FSH_ <= 24, "the bin's remaining bits resolve as 8 + 8 + (FSH_ - 16)");
     const int lane = gtid & 31, warp = gtid >> 5;
@@ -605,7 +613,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const uint32_t cnt_lo = sc.band[0], cnt_hi = sc.band[1], n_cand = sc.band[2];
     if (over > 0 || (cnt_lo > 0 && cnt_hi > 0)) {
         if (n_cand > CAND_MAX) return false;
-        redecide_band<G, WIDE, BY_POS>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r);
+        redecide_band<G, WIDE, BY_POS>(gtid, hm, sc, n_cand, cnt_hi - over, Kt_head, S_max, r, t_stride);
     }
     POST_CLK(3);
     return true;

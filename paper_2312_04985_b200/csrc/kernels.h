@@ -24,7 +24,7 @@ size_t split_scratch_bytes(int units, int S_max, int splits);
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                       const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                       int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                      int32_t* status, int splits, void* scratch, cudaStream_t stream);
+                                      int32_t* status, int splits, void* scratch, bool one_k, cudaStream_t stream);
 
 // sparq_decode_pipe.cu: persistent warp-specialised variant for S_max small enough that three key
 // buffers, the copy ring and two post-phase scratch areas fit in shared memory

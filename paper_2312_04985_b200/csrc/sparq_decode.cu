@@ -266,8 +266,12 @@ struct SplitShared {
     uint32_t band[4];
     uint32_t cnt[4];
     uint32_t ticket;
+    alignas(16) uint16_t qmask[D];   // ONE_K: q with the components outside i1 zeroed (read as 16-byte vectors)
 };
 
+// ONE_K: the variant that stores K once (no transposed copy): stage a2 reads whole rows of K, a
+// half-warp per position, and multiplies by the masked query; everything after it is unchanged.
+template <bool ONE_K>
 __global__ void __launch_bounds__(FNT, SPLIT_CTAS)
 sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                    const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
@@ -313,7 +317,7 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     PHASE_MARK(0);
 
     // ------------------------------------------------------------------ a2 (+ a3 statistics) over this CTA's slice
-    const sparq_half* Kt_head = Kt + kv_head * (size_t)D * S_max;
+    const sparq_half* Kt_head = ONE_K ? nullptr : Kt + kv_head * (size_t)D * S_max;
     uint32_t* keys = ws_keys + (size_t)bh * S_max;
     const float c1 = hm.inv_tau * LOG2E;
     uint32_t kmax = 0;
@@ -321,6 +325,51 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     __half2 mx[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) mx[e] = __float2half2_rn(0.f);
+    if constexpr (ONE_K) {
+        // the masked query, then rows of K: lane l of a half-warp owns components 8l .. 8l+7
+        if (tid < D) sh.qmask[tid] = 0;
+        __syncthreads();
+        if (tid < r) sh.qmask[hm.i1[tid]] = hm.qh[tid];
+        __syncthreads();
+        const int hw = tid >> 4, l16 = tid & 15;
+        const uint4 qm = *reinterpret_cast<const uint4*>(sh.qmask + l16 * 8);
+        const uint32_t qw[4] = {qm.x, qm.y, qm.z, qm.w};
+        const uint4* Kh = reinterpret_cast<const uint4*>(K + kv_head * (size_t)S_max * D);
+        const int n_pass = (n + SCH - 1) / SCH;
+        for (int c = p; c < n_pass; c += splits) {
+            for (int i0 = 0; i0 < SCH / (FNT / 16); i0 += 4) {           // four rows in flight per half-warp
+                uint4 v[4];
+                int t[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    t[u] = c * SCH + (i0 + u) * (FNT / 16) + hw;
+                    v[u] = t[u] < n ? ld_stream(Kh + (size_t)t[u] * (D / 8) + l16) : make_uint4(0u, 0u, 0u, 0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    float part = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        fma_h(part, (uint16_t)(qw[e] & 0xffffu), (uint16_t)(w[e] & 0xffffu));
+                        fma_h(part, (uint16_t)(qw[e] >> 16), (uint16_t)(w[e] >> 16));
+                        mx[e] = __hmax2(mx[e], __habs2(*reinterpret_cast<const __half2*>(&w[e])));
+                    }
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) part += __shfl_xor_sync(FULL, part, o, 16);
+                    if (l16 == 0 && t[u] < n) {
+                        const uint32_t kk = key32(part);
+                        keys[t[u]] = kk;
+                        kmax = max(kmax, kk);
+                        atomicAdd(&hist1[kk >> (32 - SPLIT_FB)], 1u);
+                        const float cm = part * c1;
+                        if (cm > zm) { zs *= ex2(zm - cm); zm = cm; }
+                        zs += ex2(cm - zm);
+                    }
+                }
+            }
+        }
+    } else
     {
         const uint4* Kt_vec = reinterpret_cast<const uint4*>(Kt_head);
         const int row_vecs = S_max >> 3;
@@ -417,11 +466,14 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     sc.i2 = sh.i2; sc.red = sh.red; sc.redu = sh.redu; sc.res = sh.res; sc.band = sh.band;
     const float kabs = __uint_as_float(kabs_bits);
     SelectResult sel;
-    if (!select_prefilled<FCTA, SPLIT_FB, true>(tid, hm, keys, kmax, kabs, Z, sc, hist1, r, S_max, Kt_head, sel)) {
+    // where the fp64 re-decision finds component c of position t: Kt[c * S_max + t], or K[t * d_h + c]
+    const sparq_half* band_src = ONE_K ? K + kv_head * (size_t)S_max * D : Kt_head;
+    const int c_stride = ONE_K ? 1 : S_max, t_stride = ONE_K ? D : 1;
+    if (!select_prefilled<FCTA, SPLIT_FB, true>(tid, hm, keys, kmax, kabs, Z, sc, hist1, r, c_stride, band_src, sel, t_stride)) {
 #ifdef SPARQ_PHASE_CLOCKS
         if (tid == 0) atomicAdd(&g_phase_clocks[7], 1ull);
 #endif
-        sel = select_generic<FCTA>(tid, hm, keys, kmax, kabs, sc, r, S_max, Kt_head);
+        sel = select_generic<FCTA>(tid, hm, keys, kmax, kabs, sc, r, c_stride, band_src, t_stride);
     }
     PHASE_MARK(2);
     finish<FCTA, 4>(tid, hm, keys, kmax, sel, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
@@ -488,27 +540,28 @@ size_t split_scratch_bytes(int units, int S_max, int splits) {
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                       const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                       int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                      int32_t* status, int splits, void* scratch, cudaStream_t stream) {
+                                      int32_t* status, int splits, void* scratch, bool one_k, cudaStream_t stream) {
     const int units = B * Hq;
     uint32_t* ws_keys = static_cast<uint32_t*>(scratch);
     uint32_t* ws_part = ws_keys + (size_t)units * S_max;
     uint32_t* ws_hist = ws_part + (size_t)units * splits * PART_WORDS;
     unsigned int* ws_count = ws_hist + (size_t)units * splits * SPLIT_FBINS;
     const size_t dyn = post_dynamic_smem(S_max);
-    cudaError_t e = cudaFuncSetAttribute(sparq_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    auto kernel = one_k ? sparq_split_kernel<true> : sparq_split_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     // Half of the SM's memory as shared memory holds the five CTAs; the other half stays L1, whose
     // size bounds how many of the streaming loads can be in flight (measured: 50 % beats both 62 % and
     // the driver's own choice).
-    e = cudaFuncSetAttribute(sparq_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 50);
     if (e != cudaSuccess) return e;
     if (splits > 1) {
         e = cudaMemsetAsync(ws_count, 0, (size_t)units * sizeof(unsigned int), stream);
         if (e != cudaSuccess) return e;
     }
-    sparq_split_kernel<<<dim3(splits, units), FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
-                                                                 post_bm_words(S_max), out, idx_r, idx_k, alpha, status,
-                                                                 ws_keys, ws_part, ws_hist, ws_count);
+    kernel<<<dim3(splits, units), FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
+                                                     post_bm_words(S_max), out, idx_r, idx_k, alpha, status,
+                                                     ws_keys, ws_part, ws_hist, ws_count);
     return cudaGetLastError();
 }
 

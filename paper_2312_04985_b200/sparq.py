@@ -26,7 +26,8 @@ HEAD_DIM = 128
 
 EXPORTS = ("sparq_status_string", "sparq_max_seq_len", "sparq_cache_build", "sparq_cache_append", "sparq_decode",
            "sparq_workspace_bytes", "dense_decode", "dense_workspace_bytes", "dense_decode_static", "sparq_step_host",
-           "sparq_step_host_staging_bytes", "sparq_decode_grouped", "sparq_grouped_workspace_bytes")
+           "sparq_step_host_staging_bytes", "sparq_decode_grouped", "sparq_grouped_workspace_bytes",
+           "sparq_decode_1xk", "sparq_1xk_workspace_bytes")
 
 
 class SparqError(RuntimeError):
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.sparq_decode_grouped.argtypes = [vp] * 6 + [i] * 8 + [vp] * 4 + [vp, sz, vp, vp]
         L.sparq_grouped_workspace_bytes.restype = sz
         L.sparq_grouped_workspace_bytes.argtypes = [i] * 5
+        L.sparq_decode_1xk.restype = i
+        L.sparq_decode_1xk.argtypes = [vp] * 5 + [i] * 7 + [vp] * 4 + [vp, sz, vp, vp]
+        L.sparq_1xk_workspace_bytes.restype = sz
+        L.sparq_1xk_workspace_bytes.argtypes = [i] * 5
         _lib = L
     return _lib
 
@@ -175,6 +180,26 @@ def sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, r, k, out, workspace, real
                                         0 if workspace is None else workspace.numel() * workspace.element_size(),
                                         _dev(status, torch.int32, "status"), _stream(q))
     _check("sparq_decode_grouped", rc)
+    return out
+
+
+def sparq_1xk_workspace_bytes(B, Hq, Hkv, d, S_max) -> int:
+    return int(lib().sparq_1xk_workspace_bytes(B, Hq, Hkv, d, S_max))
+
+
+def sparq_decode_1xk(q, K, V, vbar, seq_lens, r, k, out, workspace, idx_r=None, idx_k=None, alpha=None, status=None):
+    B, Hq, d = q.shape
+    Hkv, S_max = K.shape[1], K.shape[2]
+    with torch.cuda.device(q.device):
+        rc = lib().sparq_decode_1xk(_dev(q, torch.float16, "q"), _dev(K, torch.float16, "K"), _dev(V, torch.float16, "V"),
+                                    _dev(vbar, torch.float16, "vbar"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                    B, Hq, Hkv, d, S_max, int(r), int(k), _dev(out, torch.float16, "out"),
+                                    _dev(idx_r, torch.int32, "idx_r"), _dev(idx_k, torch.int32, "idx_k"),
+                                    _dev(alpha, torch.float32, "alpha"),
+                                    None if workspace is None else workspace.data_ptr(),
+                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _dev(status, torch.int32, "status"), _stream(q))
+    _check("sparq_decode_1xk", rc)
     return out
 
 
