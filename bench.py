@@ -357,6 +357,38 @@ def run_b200(args):
         grouped = {"us": g_us, "compulsory_bytes": g_bytes, "hbm_gbs_compulsory": g_bytes / (g_us * 1e-6) / 1e9,
                    "speedup_vs_dense": dense_us / g_us, "speedup_vs_per_head": sparq_full_us / g_us}
 
+    # ---------------------------------------------------------------- the same step replayed from CUDA graphs
+    # (one captured append + decode per cache copy; the lengths advance on the device, so a replay is a step)
+    for c in caches:
+        c.to_start()
+    graphs = []
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for c in caches:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side), torch.cuda.graph(g, stream=side):
+            sparq.sparq_cache_append(pool["k_new"][0], pool["v_new"][0], c.K, c.Kt, c.V, c.vsum, c.vbar, c.seq_lens, status)
+            sparq.sparq_decode(pool["q"][0], c.K, c.Kt, c.V, c.vbar, c.seq_lens, r, k, out, workspace=dec_ws, status=status)
+        graphs.append(g)
+    torch.cuda.synchronize()
+
+    def graph_step(i):
+        if (i // n_copies) % period == 0:
+            caches[i % n_copies].rewind()
+        graphs[i % n_copies].replay()
+
+    for i in range(3 * n_copies):
+        graph_step(i)
+    barrier()
+    g_steps = min(args.steps, 2 * period * n_copies)
+    t_beg.record()
+    for i in range(g_steps):
+        graph_step(i)
+    t_end.record()
+    barrier()
+    graph_us = max_over_ranks(1e3 * t_beg.elapsed_time(t_end) / g_steps)
+    del graphs
+
     # ---------------------------------------------------------------- end to end from host buffers
     staging = torch.empty(sparq.sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k), dtype=torch.uint8, device=dev)
     hq = [pool["q"][j].cpu().pin_memory() for j in range(POOL)]
@@ -420,7 +452,7 @@ def run_b200(args):
                          % ("inputs larger than L2" if n_copies == 1 else "steps rotate over independent cache copies larger than L2 together",
                             cache_bytes / 1e9, n_copies, "y" if n_copies == 1 else "ies", POOL),
                    "parallelism": "independent batches per GPU, no collective"},
-        "us_per_step": us_per_step, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
+        "us_per_step": us_per_step, "graph_replay_us_per_step": graph_us, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
         "dense_decode_us": dense_us, "speedup_vs_dense": dense_us / sparq_full_us, "sparq_decode_grouped": grouped,
         "sparq_decode_1xk": one_k,
         "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, end_mean, d) / (dense_us * 1e-6) / 1e9,

@@ -32,6 +32,17 @@ constexpr int GFB = 11;                  // first digit of the selection keys
 constexpr int GFBINS = 1 << GFB;
 using CTA = Group<NT, 0>;
 
+// Optional per-stage cycle counters (thread 0 of every CTA, summed); compiled in only with
+// -DSPARQ_PHASE_CLOCKS for tuning, never in the shipped library.
+#ifdef SPARQ_PHASE_CLOCKS
+__device__ unsigned long long g_group_clocks[16];
+#define GCLK_INIT() long long gc_prev_ = clock64()
+#define GCLK(i) do { if (threadIdx.x == 0) { long long gc_now_ = clock64(); atomicAdd(&g_group_clocks[i], (unsigned long long)(gc_now_ - gc_prev_)); gc_prev_ = gc_now_; } } while (0)
+#else
+#define GCLK_INIT()
+#define GCLK(i)
+#endif
+
 struct GroupShared {
     HeadMeta hm;                          // the head being finished (g5); i1 and n are the group's
     int32_t i2[SPARQ_K_MAX];
@@ -94,6 +105,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         return;
     }
     const int k_eff = min(k, n);
+    GCLK_INIT();
     for (int i = tid; i < GFBINS / 4; i += NT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
 
     // ------------------------------------------------------------------ g1: group top-r, per-head tau
@@ -151,6 +163,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         return;
     }
 
+    GCLK(0);
     // ------------------------------------------------------------------ g2: one stream for the whole group
     const sparq_half* Kt_head = Kt + (size_t)bk * D * S_max;
     uint32_t* ws_unit = ws + (size_t)bk * (G + 1) * S_max;                // [G][S_max] chains, then [S_max] selection keys
@@ -201,6 +214,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
             *reinterpret_cast<uint4*>(dst + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
         }
     }
+    GCLK(1);
     // per head: the CTA-wide maximum and the denominator relative to it
     float inv_z[G], vmax[G];
 #pragma unroll
@@ -239,6 +253,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
 #pragma unroll
     for (int h = 0; h < G; ++h) { vmax[h] = unkey32(sh.kmax[h]); inv_z[h] = 1.0f / sh.zsum[h]; }
 
+    GCLK(2);
     // ------------------------------------------------------------------ g3: summed scores as selection keys
     uint32_t smax = 0;
     for (int c = 0; c < n_pass; ++c) {                       // every position of the group, whoever streamed it
@@ -270,6 +285,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         group_max2_u32<CTA>(smax, dummy, sh.redu, tid);      // barriers: histogram and selection keys complete
     }
 
+    GCLK(3);
     // ------------------------------------------------------------------ g4: top-k of the summed scores
     PostScratch sc;
     carve_post_scratch(sc, dyn_smem, CTA::NHW, bm_words);
@@ -279,6 +295,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     if (!select_prefilled<CTA, GFB, true, true>(tid, hm, keys_sum, smax, 0.f, 1.f, sc, hist1, r, S_max, Kt_head, sel_res))
         sel_res = select_generic<CTA, true>(tid, hm, keys_sum, smax, 0.f, sc, r, S_max, Kt_head);
 
+    GCLK(4);
     // ------------------------------------------------------------------ g5: per head alpha, attention, Step 3
     const sparq_half* K_head = K + (size_t)bk * S_max * D;
     const sparq_half* V_head = V + (size_t)bk * S_max * D;
@@ -299,6 +316,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
                        out0 + (size_t)h * D, (h == 0 && idx_k) ? idx_k + (size_t)bk * k : nullptr,
                        alpha0 ? alpha0 + h : nullptr, /*build_list=*/h == 0, /*realloc=*/realloc != 0);
     }
+    GCLK(5);
 }
 
 int grouped_bm_words(int S_max) { return (S_max + 127) / 128 * 4; }
@@ -325,6 +343,15 @@ cudaError_t launch_g(const sparq_half* q, const sparq_half* K, const sparq_half*
 }
 
 }  // namespace
+
+#ifdef SPARQ_PHASE_CLOCKS
+extern "C" int sparq_debug_group_clocks(unsigned long long* out16, int reset) {
+    cudaDeviceSynchronize();
+    if (out16 && cudaMemcpyFromSymbol(out16, g_group_clocks, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+    if (reset) { unsigned long long z[16] = {0}; if (cudaMemcpyToSymbol(g_group_clocks, z, sizeof(z)) != cudaSuccess) return 1; }
+    return 0;
+}
+#endif
 
 size_t grouped_dynamic_smem(int S_max) { return (post_scratch_bytes(CTA::NHW, grouped_bm_words(S_max)) + 127) & ~(size_t)127; }
 
