@@ -251,7 +251,8 @@ def dense_decode(q, K, V, seq_lens):
 # Step 3 is applied per head, or left out (``realloc=False``: the paper dropped it for its
 # grouped-query models).  Readings: ties go to the smaller index in both selections; the Step 2
 # selection is on the summed softmax scores themselves (a sum over heads does not commute with the
-# softmax, so the logits cannot stand in for them here).
+# softmax, so the logits cannot stand in for them here), ranked through the logarithm of the sum so
+# that scores below the floating-point range still rank by their size instead of tying at zero.
 def group_top_r(Q: np.ndarray, r: int):
     """Step 1 for a group: Q [g, d_h]; the r largest components of sum_h |Q[h]|.
     Returns (i1 ascending, relative gap at the boundary)."""
@@ -265,33 +266,44 @@ def group_top_r(Q: np.ndarray, r: int):
     return np.sort(order[:r]).astype(np.int64), gap
 
 
+def log_softmax(x: np.ndarray) -> np.ndarray:
+    """log of :func:`softmax`, without forming the exponentials of far-away entries."""
+    x = np.asarray(x, dtype=F64)
+    m = np.max(x)
+    return x - (m + math.log(float(np.sum(np.exp(x - m)))))
+
+
 def group_scores(Q: np.ndarray, K: np.ndarray, i1: np.ndarray, n: int):
     """Eq. (7) for every head of the group over the shared component set i1: returns
-    (s_hat [g, n], tau [g]); tau is Eq. (9) per query head."""
+    (log s_hat [g, n], tau [g]); tau is Eq. (9) per query head.  The scores are kept as their
+    logarithms: exp() of them is s_hat, and entries far below the largest one, which would
+    underflow to equal zeros, keep their order."""
     Q = np.asarray(Q, dtype=F64)
     g = Q.shape[0]
-    s_hat = np.zeros((g, n), dtype=F64)
+    log_s = np.zeros((g, n), dtype=F64)
     tau = np.zeros(g, dtype=F64)
     for h in range(g):
         l_hat, tau[h] = approx_logits_fast(Q[h], K, i1, n)
-        s_hat[h] = softmax(l_hat)
-    return s_hat, tau
+        log_s[h] = log_softmax(l_hat)
+    return log_s, tau
 
 
-def group_top_k(s_hat: np.ndarray, k: int):
+def group_top_k(log_s: np.ndarray, k: int):
     """Step 2 for a group: the min(k, n) positions with the largest sum_h s_hat[h, t] (ties to the
-    smaller position), ascending; alpha [g] = each head's own score mass on that set (Step 3);
-    relative gap of the summed scores at the boundary."""
-    s_hat = np.asarray(s_hat, dtype=F64)
-    g, n = s_hat.shape
+    smaller position), ascending; alpha [g] = each head's own score mass on that set (Step 3).
+    The sums are ranked through their logarithms, log sum_h exp(log_s[h, t]) (same order, no
+    underflow); ``gap`` is the difference of that logarithm between the last selected and the
+    first rejected position (for small values: the relative gap of the summed scores)."""
+    log_s = np.asarray(log_s, dtype=F64)
+    g, n = log_s.shape
     k_eff = max(0, min(int(k), n))
     if k_eff == 0:
         return np.zeros(0, dtype=np.int64), np.zeros(g, dtype=F64), math.inf
-    total = np.sum(s_hat, axis=0)
-    order = _desc_order(total)
+    log_total = np.logaddexp.reduce(log_s, axis=0)
+    order = _desc_order(log_total)
     sel = np.sort(order[:k_eff]).astype(np.int64)
-    alpha = np.sum(s_hat[:, sel], axis=1)
-    gap = math.inf if k_eff == n else _rel_gap(total[order[k_eff - 1]], total[order[k_eff]])
+    alpha = np.sum(np.exp(log_s[:, sel]), axis=1)
+    gap = math.inf if k_eff == n else abs(float(log_total[order[k_eff - 1]] - log_total[order[k_eff]]))
     return sel, alpha, gap
 
 
@@ -310,10 +322,10 @@ def group_from_i2(Q, K, V, v_bar, i2, alpha, realloc=True):
 
 
 def group_from_i1(Q, K, V, v_bar, n, i1, k, realloc=True):
-    s_hat, tau = group_scores(Q, K, np.asarray(i1, dtype=np.int64), n)
-    i2, alpha, gap_k = group_top_k(s_hat, k)
+    log_s, tau = group_scores(Q, K, np.asarray(i1, dtype=np.int64), n)
+    i2, alpha, gap_k = group_top_k(log_s, k)
     out = group_from_i2(Q, K, V, v_bar, i2, alpha, realloc)
-    return dict(out=out, i2=i2, alpha=alpha, gap_k=gap_k, tau=tau, s_hat=s_hat)
+    return dict(out=out, i2=i2, alpha=alpha, gap_k=gap_k, tau=tau, log_s=log_s)
 
 
 def sparq_group(Q, K, V, v_bar, n, r, k, realloc=True):

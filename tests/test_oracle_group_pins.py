@@ -67,9 +67,12 @@ def test_step2_brute_force_maximises_the_groups_total_mass():
         k, r = int(RNG.integers(1, n)), int(RNG.integers(1, 9))
         Q, K, V = rand_group(g, n, d=8)
         i1, _ = O.group_top_r(Q, r)
-        s_hat, tau = O.group_scores(Q, K, i1, n)
+        log_s, tau = O.group_scores(Q, K, i1, n)
+        s_hat = np.exp(log_s)
         np.testing.assert_allclose(s_hat.sum(axis=1), 1.0, rtol=1e-13)
-        i2, alpha, _ = O.group_top_k(s_hat, k)
+        for h in range(g):                                    # the kept logarithms are those of Eq. (7)'s softmax
+            np.testing.assert_allclose(s_hat[h], O.softmax(O.approx_logits(Q[h], K, i1, n)[0]), rtol=1e-12)
+        i2, alpha, _ = O.group_top_k(log_s, k)
         best = max(itertools.combinations(range(n), k), key=lambda S: s_hat[:, list(S)].sum())
         assert sorted(best) == i2.tolist()
         for h in range(g):
@@ -130,13 +133,28 @@ def test_heads_disagree_and_the_sum_decides():
     K = np.array([[4.0, 0.0], [0.0, 4.0], [3.4, 3.4]])
     Q = np.array([[1.0, 0.0], [0.0, 1.0]])
     V = np.eye(3, 2)
-    s_hat, _ = O.group_scores(Q, K, np.array([0, 1]), 3)
-    assert int(np.argmax(s_hat[0])) == 0 and int(np.argmax(s_hat[1])) == 1
-    i2, alpha, _ = O.group_top_k(s_hat, 1)
+    log_s, _ = O.group_scores(Q, K, np.array([0, 1]), 3)
+    assert int(np.argmax(log_s[0])) == 0 and int(np.argmax(log_s[1])) == 1
+    i2, alpha, _ = O.group_top_k(log_s, 1)
     assert i2.tolist() == [2]
     # by hand: tau = sqrt(2 * 1/1); head 0 logits (4, 0, 3.4)/sqrt 2
     e = np.exp(np.array([4.0, 0.0, 3.4]) / math.sqrt(2.0))
     assert alpha[0] == pytest.approx(e[2] / e.sum(), rel=1e-13)
+
+
+def test_scores_below_the_floating_point_range_still_rank_by_size():
+    """Keys so spread out that most softmax scores underflow even in float64: the selection must
+    still follow the scores' order (here: the logits' order, the group being one head), not the
+    positions' order among equal zeros."""
+    n, d = 40, 8
+    q = np.zeros(d); q[0] = 1.0
+    K = np.zeros((n, d)); K[:, 0] = np.linspace(0.0, 4000.0, n)[::-1].copy()      # logits 4000/sqrt(8) apart overall
+    K[[3, 17]] = K[[17, 3]]
+    V = RNG.standard_normal((n, d))
+    res = O.sparq_group(q[None], K, V, O.mean_value(V, n), n, 1, 10)
+    want = np.sort(np.argsort(-K[:, 0], kind="stable")[:10])
+    assert res["i2"].tolist() == want.tolist()
+    assert np.exp(res["log_s"][0]).min() == 0.0               # the scores themselves do underflow
 
 
 def test_batched_grouped_decode_maps_consecutive_heads_to_a_kv_head():
