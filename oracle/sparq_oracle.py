@@ -73,9 +73,13 @@ def temperature(q: np.ndarray, i1: np.ndarray) -> float:
     """Eq. (9): tau = sqrt(d_h * ||q o m_q||_1 / ||q||_1), per query head."""
     q = np.asarray(q, dtype=F64)
     total = float(np.sum(np.abs(q)))
-    if total == 0.0:
+    kept = float(np.sum(np.abs(q[i1])))
+    if total == 0.0 or kept == 0.0:
+        # every approximate logit is 0 whatever tau is (reading: tau := 1, uniform s_hat).  With a
+        # head's own top-r this needs q = 0; with a component set chosen by a group (below) a head
+        # can have all of its weight outside it.
         return 1.0
-    return math.sqrt(q.shape[0] * float(np.sum(np.abs(q[i1]))) / total)
+    return math.sqrt(q.shape[0] * kept / total)
 
 
 def approx_logits(q: np.ndarray, K: np.ndarray, i1: np.ndarray, n: int):

@@ -11,15 +11,17 @@
 //       chains of exact fp16 x fp16 products.  The chains go to a scratch buffer as order-preserving
 //       keys (g x 4 bytes per position); each head's maximum and softmax denominator are
 //       accumulated on the way (online, per thread)                                    (Eq. (7))
-//   g3  every thread reads its own positions back, forms sum_h s_hat[h, t] and writes it as the
-//       position's selection key, filling the histogram of the keys' top bits
+//   g3  every thread reads the chains back, forms log2 sum_h s_hat[h, t] (a log-sum-exp: scores below
+//       fp32's range keep their order) and writes it as the position's selection key, filling the
+//       histogram of the keys' top bits
 //   g4  top-k of the summed scores (decode_common.cuh; equal keys go to the lowest positions)
 //   g5  per head: alpha, gather of the k selected K/V rows (from L1/L2 after the first head),
 //       exact attention, Step 3 (or not)                                        (Eqs. (8), (10))
 //
-// The summed scores are sums of fp32 exponentials, so unlike the per-head path the selection is not
-// re-decided in fp64: positions whose summed scores differ by less than the fp32 evaluation error
-// (about 1e-5 relative, bounded by 1e-4) may swap against a float64 evaluation.
+// The summed scores are evaluated in fp32, so unlike the per-head path the selection is not re-decided
+// in fp64: positions whose summed scores differ by less than the fp32 evaluation error (the chains'
+// rounding bound over tau plus a few ulps of the logit's distance from the maximum) may swap against a
+// float64 evaluation.
 #include "decode_common.cuh"
 #include "kernels.h"
 
@@ -149,7 +151,8 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         if (tid >= r && tid < r_pad) sh.qh[h][tid] = 0;
         float l1_all = aq[h], l1_sel = sel ? aq[h] : 0.f;
         group_sum2<CTA>(l1_all, l1_sel, sh.red, tid);
-        if (tid == 0) sh.inv_tau[h] = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
+        // (a head with no weight on the group's components has all-zero approximate logits: tau := 1)
+        if (tid == 0) sh.inv_tau[h] = (l1_all > 0.f && l1_sel > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
     }
     if (tid == 0) { hm.bh = bk; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; hm.l1_sel = 0.f; }
     __syncthreads();
@@ -216,7 +219,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     }
     GCLK(1);
     // per head: the CTA-wide maximum and the denominator relative to it
-    float inv_z[G], vmax[G];
+    float lz[G], vmax[G];                                    // per head: log2 of the denominator, the largest chain
 #pragma unroll
     for (int h = 0; h < G; ++h) {
         uint32_t km = kmx[h], dummy = 0;
@@ -251,7 +254,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     }
     __syncthreads();
 #pragma unroll
-    for (int h = 0; h < G; ++h) { vmax[h] = unkey32(sh.kmax[h]); inv_z[h] = 1.0f / sh.zsum[h]; }
+    for (int h = 0; h < G; ++h) { vmax[h] = unkey32(sh.kmax[h]); lz[h] = __log2f(sh.zsum[h]); }
 
     GCLK(2);
     // ------------------------------------------------------------------ g3: summed scores as selection keys
@@ -260,16 +263,31 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         const int t0 = c * CHG + tid * 8;
         const int nvalid = min(8, n - t0);
         if (nvalid <= 0) continue;
-        float ssum[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) ssum[e] = 0.f;
+        // log2 of the summed scores: x_h = log2 s_hat[h, t], then max_h x_h + log2 sum_h 2^(x_h - max).  Ranking
+        // the logarithm keeps the order of scores that would underflow as plain exponentials; for a group
+        // of one it is the logit itself.
+        float x[G][8], ssum[8];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
             const uint32_t* src = ws_unit + (size_t)h * S_max + t0;
             const uint4 a = __ldcg(reinterpret_cast<const uint4*>(src)), bq = __ldcg(reinterpret_cast<const uint4*>(src + 4));
             const uint32_t kk[8] = {a.x, a.y, a.z, a.w, bq.x, bq.y, bq.z, bq.w};
 #pragma unroll
-            for (int e = 0; e < 8; ++e) ssum[e] += ex2((unkey32(kk[e]) - vmax[h]) * c1[h]) * inv_z[h];
+            for (int e = 0; e < 8; ++e) x[h][e] = (unkey32(kk[e]) - vmax[h]) * c1[h] - lz[h];
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float mxe = x[0][e];
+#pragma unroll
+            for (int h = 1; h < G; ++h) mxe = fmaxf(mxe, x[h][e]);
+            if constexpr (G == 1) {
+                ssum[e] = mxe;
+            } else {
+                float acc2 = 0.f;
+#pragma unroll
+                for (int h = 0; h < G; ++h) acc2 += ex2(x[h][e] - mxe);
+                ssum[e] = mxe + __log2f(acc2);
+            }
         }
         uint32_t ks[8];
 #pragma unroll

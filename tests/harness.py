@@ -152,7 +152,7 @@ def oracle_all_units(q, K, V, seq, r, k):
 def flat(gpu):
     d = {}
     for key, v in gpu.items():
-        d[key] = v.reshape(-1, v.shape[-1]) if v.ndim == 3 else v.reshape(-1)
+        d[key] = v.reshape(v.shape[0] * v.shape[1], v.shape[-1]) if v.ndim == 3 else v.reshape(-1)
     return d
 
 

@@ -157,6 +157,21 @@ def test_scores_below_the_floating_point_range_still_rank_by_size():
     assert np.exp(res["log_s"][0]).min() == 0.0               # the scores themselves do underflow
 
 
+def test_head_with_no_weight_on_the_groups_components_scores_uniformly():
+    """The group's top-r can miss every non-zero component of one head: that head's approximate
+    logits are all 0, its s_hat uniform (tau := 1), and it does not sway the group's selection."""
+    n, d = 12, 6
+    Q = np.zeros((2, d)); Q[0, 0] = 3.0; Q[1, 5] = 1.0
+    K = RNG.standard_normal((n, d)); V = RNG.standard_normal((n, d))
+    i1, _ = O.group_top_r(Q, 1)
+    assert i1.tolist() == [0]
+    log_s, tau = O.group_scores(Q, K, i1, n)
+    assert tau[1] == 1.0 and np.allclose(np.exp(log_s[1]), 1.0 / n)
+    res = O.sparq_group(Q, K, V, O.mean_value(V, n), n, 1, 4)
+    assert res["i2"].tolist() == O.sparq_head(Q[0], K, V, O.mean_value(V, n), n, 1, 4)["i2"].tolist()
+    assert res["alpha"][1] == pytest.approx(4.0 / n) and np.isfinite(res["out"]).all()
+
+
 def test_batched_grouped_decode_maps_consecutive_heads_to_a_kv_head():
     B, Hq, Hkv, n, d = 2, 6, 2, 20, 16
     q = RNG.standard_normal((B, Hq, d))
