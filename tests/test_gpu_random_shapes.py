@@ -71,3 +71,46 @@ def test_random_shape(seed):
         compare_groups(run_grouped(cache, q, r, k, realloc=realloc), qn, Knp, Vnp, seq.numpy(), r, k, realloc=realloc,
                        what=what + " grouped")
     cache.check_status(0)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_append_sequences(seed):
+    """Random start lengths, a random number of appends (crossing 16-byte vector boundaries of Kt, up
+    to a full cache), then the layout invariants and a decode against the oracle."""
+    rng = np.random.default_rng(5000 + seed)
+    B, Hkv = int(rng.integers(1, 5)), int(rng.integers(1, 5))
+    g = int(rng.choice([1, 2, 4]))
+    Hq = Hkv * g
+    S = int(rng.choice([16, 40, 128, 264, 1032]))
+    T = int(rng.integers(1, min(24, S)))
+    start = rng.integers(0, S - T + 1, size=B)
+    if seed % 2 == 0:
+        start[0] = S - T                                      # this one ends exactly full
+    gen = torch.Generator().manual_seed(seed)
+    K = torch.randn(B, Hkv, S, 128, generator=gen).half()
+    V = torch.randn(B, Hkv, S, 128, generator=gen).half()
+    q = torch.randn(B, Hq, 128, generator=gen).half()
+    seq0 = torch.tensor(start, dtype=torch.int32)             # (a start of 0 is an empty sequence: sparq_cache_build takes it)
+    cache = H.DeviceCache(K, V, seq0)
+    for i in range(T):
+        idx = (seq0.long() + i).view(B, 1, 1, 1).expand(B, Hkv, 1, 128)
+        cache.append(torch.gather(K, 2, idx).squeeze(2).contiguous(), torch.gather(V, 2, idx).squeeze(2).contiguous())
+    torch.cuda.synchronize()
+    cache.check_status(0)
+    Kt = cache.Kt.cpu()
+    for b in range(B):
+        n = int(seq0[b]) + T
+        assert int(cache.seq_lens[b]) == n
+        assert torch.equal(cache.K[b, :, :n].cpu(), K[b, :, :n]) and torch.equal(cache.V[b, :, :n].cpu(), V[b, :, :n])
+        assert torch.equal(Kt[b, :, :, :n], K[b, :, :n].transpose(1, 2))
+        n8 = (n + 7) // 8 * 8
+        assert (Kt[b, :, :, n:n8] == 0).all(), "zeros up to the end of the last 16-byte vector"
+        vb = V[b, :, :n].double().mean(dim=1)
+        np.testing.assert_allclose(cache.vbar[b].cpu().double().numpy(), vb.numpy(), atol=2e-3)
+    seq = seq0 + T
+    r, k = int(rng.choice([4, 16, 32])), int(rng.choice([1, 8, 64]))
+    ora = c_oracle.sparq_decode(q.numpy(), K.numpy(), V.numpy(), seq.numpy(), r, k)
+    gpu = H.flat(cache.decode(q, r, k))
+    Knp, Vnp, qn = K.numpy(), V.numpy(), q.numpy()
+    H.compare_units(gpu, ora, qn.reshape(B * Hq, -1), lambda u: Knp[u // Hq, (u % Hq) // g],
+                    lambda u: Vnp[u // Hq, (u % Hq) // g], np.repeat(seq.numpy(), Hq), r, k, "append sweep %d" % seed)
