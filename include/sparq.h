@@ -32,6 +32,8 @@
  *         seq_lens (int32)   [B]     number of valid positions of sequence b
  *     Query head h reads KV head h / (Hq / Hkv): consecutive query heads share a KV head
  *     (Section 4, "Grouped query attention").  Each query head selects its own i1 and i2.
+ *   - Every fp16 / fp32 tensor pointer and every workspace must be 16-byte aligned (the kernels use
+ *     128-bit accesses); a pointer that is not is refused with SPARQ_ERR_ALIGNMENT on the host.
  *   - Supported shapes: d == 128; Hq a multiple of Hkv; S_max a multiple of 8 (rows of Kt
  *     are then 16-byte aligned); 1 <= r <= d; 0 <= k <= SPARQ_K_MAX.
  *   - Return value: SPARQ_OK, or a SPARQ_ERR_* code for anything the host can see; in that
@@ -69,6 +71,7 @@ enum {
     SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds sparq_max_seq_len() (or, with a workspace,
                                     SPARQ_S_MAX_WORKSPACE)                                      */
     SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
+    SPARQ_ERR_ALIGNMENT = 8,     /* a tensor or workspace pointer is not 16-byte aligned          */
     SPARQ_ERR_STATIC_SCRATCH = 7,/* the problem needs more scratch than the library's fixed
                                     SPARQ_STATIC_SCRATCH_BYTES: use the call that takes a workspace */
     SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */

@@ -44,6 +44,12 @@ constexpr size_t SPARQ_PIPE_WORKSPACE_BYTES = 64;
 
 int rc(cudaError_t e) { return e == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA; }
 
+// true when any of the given pointers (NULL allowed: optional arguments) is not 16-byte aligned
+template <class... P>
+bool misaligned(P... ptrs) {
+    return (((reinterpret_cast<uintptr_t>((const void*)ptrs) & 15u) != 0) || ...);
+}
+
 }  // namespace
 
 extern "C" {
@@ -58,6 +64,7 @@ const char* sparq_status_string(int code) {
         case SPARQ_ERR_TOO_LONG: return "SPARQ_ERR_TOO_LONG";
         case SPARQ_ERR_CUDA: return "SPARQ_ERR_CUDA";
         case SPARQ_ERR_STATIC_SCRATCH: return "SPARQ_ERR_STATIC_SCRATCH";
+        case SPARQ_ERR_ALIGNMENT: return "SPARQ_ERR_ALIGNMENT";
         case SPARQ_DEV_BAD_SEQ_LEN: return "SPARQ_DEV_BAD_SEQ_LEN";
         case SPARQ_DEV_CACHE_FULL: return "SPARQ_DEV_CACHE_FULL";
         case SPARQ_DEV_TIMEOUT: return "SPARQ_DEV_TIMEOUT";
@@ -78,6 +85,7 @@ int sparq_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* s
                       int B, int Hkv, int d, int S_max, int32_t* status, void* stream) {
     if (!K || !V || !seq_lens || !Kt || !vsum || !vbar) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hkv, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (misaligned(K, V, Kt, vsum, vbar)) return SPARQ_ERR_ALIGNMENT;
     return rc(launch_cache_build(K, V, seq_lens, Kt, vsum, vbar, B, Hkv, S_max, status, (cudaStream_t)stream));
 }
 
@@ -86,6 +94,7 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
                        int32_t* seq_lens, int B, int Hkv, int d, int S_max, int32_t* status, void* stream) {
     if (!k_new || !v_new || !K || !Kt || !V || !vsum || !vbar || !seq_lens) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hkv, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (misaligned(k_new, v_new, K, Kt, V, vsum, vbar)) return SPARQ_ERR_ALIGNMENT;
     return rc(launch_cache_append(k_new, v_new, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, S_max, status,
                                   (cudaStream_t)stream));
 }
@@ -118,6 +127,7 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
+    if (misaligned(q, K, Kt, V, vbar, out, workspace)) return SPARQ_ERR_ALIGNMENT;
     const int plan = forced_plan();
     const int n_sm = device_sm_count();
     const int splits = S_max <= SPARQ_S_MAX_WORKSPACE ? split_count(B * Hq, S_max, n_sm) : 0;
@@ -162,10 +172,9 @@ int sparq_decode_1xk(const sparq_half* q, const sparq_half* K, const sparq_half*
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
     if (S_max > SPARQ_S_MAX_WORKSPACE) return SPARQ_ERR_TOO_LONG;
+    if (misaligned(q, K, V, vbar, out, workspace)) return SPARQ_ERR_ALIGNMENT;
     const int splits = one_k_splits(B * Hq, S_max);
-    if (!workspace || workspace_bytes < split_scratch_bytes(B * Hq, S_max, splits) ||
-        reinterpret_cast<uintptr_t>(workspace) % 16 != 0)
-        return SPARQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < split_scratch_bytes(B * Hq, S_max, splits)) return SPARQ_ERR_WORKSPACE;
     return rc(launch_sparq_decode_split(q, K, nullptr, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
                                         status, splits, workspace, true, (cudaStream_t)stream));
 }
@@ -185,11 +194,10 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
     const int g = Hq / Hkv;
     if (g != 1 && g != 2 && g != 4 && g != 8) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
+    if (misaligned(q, K, Kt, V, vbar, out, workspace)) return SPARQ_ERR_ALIGNMENT;
     if (S_max > SPARQ_S_MAX_WORKSPACE || grouped_dynamic_smem(S_max) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
     const int slices = grouped_slices(B * Hkv, S_max, device_sm_count());
-    if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices) ||
-        reinterpret_cast<uintptr_t>(workspace) % 16 != 0)
-        return SPARQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices)) return SPARQ_ERR_WORKSPACE;
     return rc(launch_sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, realloc, out, idx_r, idx_k,
                                           alpha, status, workspace, slices, (cudaStream_t)stream));
 }
@@ -204,6 +212,7 @@ int dense_decode(const sparq_half* q, const sparq_half* K, const sparq_half* V, 
                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
     if (!q || !K || !V || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (misaligned(q, K, V, out, workspace)) return SPARQ_ERR_ALIGNMENT;
     const size_t need = dense_scratch_bytes(B, Hq, Hkv, S_max);
     if (need && (!workspace || workspace_bytes < need)) return SPARQ_ERR_WORKSPACE;
     return rc(launch_dense_decode(q, K, V, seq_lens, B, Hq, Hkv, S_max, out, (float*)workspace, status,
@@ -214,6 +223,7 @@ int dense_decode_static(const sparq_half* q, const sparq_half* K, const sparq_ha
                         int B, int Hq, int Hkv, int d, int S_max, sparq_half* out, int32_t* status, void* stream) {
     if (!q || !K || !V || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
+    if (misaligned(q, K, V, out)) return SPARQ_ERR_ALIGNMENT;
     if (dense_scratch_bytes(B, Hq, Hkv, S_max) > SPARQ_STATIC_SCRATCH_BYTES) return SPARQ_ERR_STATIC_SCRATCH;
     float* scratch = nullptr;
     size_t bytes = 0;
@@ -238,6 +248,7 @@ int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, cons
     if (!q_host || !k_new_host || !v_new_host || !out_host) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (!staging || staging_bytes < sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k)) return SPARQ_ERR_WORKSPACE;
+    if (misaligned(staging)) return SPARQ_ERR_ALIGNMENT;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t nq = (size_t)B * Hq * d, nkv = (size_t)B * Hkv * d;
     sparq_half* q_dev = (sparq_half*)staging;

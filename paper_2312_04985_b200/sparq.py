@@ -19,6 +19,7 @@ from . import build as _build
 
 OK = 0
 ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_BAD_RK, ERR_WORKSPACE, ERR_TOO_LONG, ERR_CUDA, ERR_STATIC_SCRATCH = 1, 2, 3, 4, 5, 6, 7
+ERR_ALIGNMENT = 8
 STATIC_SCRATCH_BYTES = 8 << 20
 DEV_BAD_SEQ_LEN, DEV_CACHE_FULL, DEV_TIMEOUT = 16, 17, 18
 K_MAX = 1024

@@ -36,6 +36,7 @@ def test_every_declared_function_is_exported(lib):
 def test_status_strings(lib):
     codes = {0: "SPARQ_OK", 1: "SPARQ_ERR_NULL_POINTER", 2: "SPARQ_ERR_BAD_SHAPE", 3: "SPARQ_ERR_BAD_RK",
              4: "SPARQ_ERR_WORKSPACE", 5: "SPARQ_ERR_TOO_LONG", 6: "SPARQ_ERR_CUDA", 7: "SPARQ_ERR_STATIC_SCRATCH",
+             8: "SPARQ_ERR_ALIGNMENT",
              16: "SPARQ_DEV_BAD_SEQ_LEN", 17: "SPARQ_DEV_CACHE_FULL", 18: "SPARQ_DEV_TIMEOUT"}
     for code, name in codes.items():
         assert sparq.status_string(code) == name
@@ -58,6 +59,15 @@ def test_host_visible_errors_need_no_device(lib):
     # r and k ranges
     for r, k in ((0, 1), (129, 1), (4, -1), (4, sparq.K_MAX + 1)):
         assert lib.sparq_decode(one, one, one, one, one, one, 1, 1, 1, 128, 8, r, k, one, n, n, n, n, 0, n, n) == sparq.ERR_BAD_RK
+    # a tensor pointer that is not 16-byte aligned (the kernels would fault on it)
+    odd = ctypes.c_void_p(24)
+    assert lib.sparq_decode(one, one, odd, one, one, one, 1, 1, 1, 128, 8, 1, 1, one, n, n, n, n, 0, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.sparq_decode(one, one, one, one, one, one, 1, 1, 1, 128, 8, 1, 1, one, n, n, n, odd, 64, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.sparq_cache_append(odd, one, one, one, one, one, one, one, 1, 1, 128, 8, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.sparq_cache_build(one, one, one, one, odd, one, 1, 1, 128, 8, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.dense_decode(one, one, one, one, 1, 1, 1, 128, 8, odd, n, 0, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.sparq_decode_grouped(one, one, one, one, one, one, 1, 2, 1, 128, 8, 1, 1, 1, odd, n, n, n, one, 1 << 20, n, n) == sparq.ERR_ALIGNMENT
+    assert lib.sparq_decode_1xk(one, odd, one, one, one, 1, 1, 1, 128, 8, 1, 1, one, n, n, n, one, 1 << 20, n, n) == sparq.ERR_ALIGNMENT
     # dense_decode: a split plan without a workspace; the static variant: a plan beyond its built-in scratch
     assert sparq.dense_workspace_bytes(1, 32, 32, 128, 4096) == 32 * 16 * 130 * 4   # 16 splits of 256 positions
     assert lib.dense_decode(one, one, one, one, 1, 32, 32, 128, 4096, one, n, 0, n, n) == sparq.ERR_WORKSPACE
