@@ -28,9 +28,9 @@ int device_sm_count() {
 }
 
 // SPARQ_DECODE_PLAN=simple|pipe|split forces one of the sparq_decode plans (tests and tuning).
-// Unset or anything else: the split-S plan when there are fewer units than SMs and the caller
-// passed its workspace, else the persistent pipelined kernel whenever its buffers fit, else one
-// CTA per unit.
+// Unset or anything else: the persistent pipelined kernel whenever one unit's keys fit its shared
+// memory, except for fewer units than SMs with a lot to stream each; otherwise -- and for caches
+// too long for it -- the split plan if the caller passed its workspace; else one CTA per unit.
 int forced_plan() {
     const char* e = getenv("SPARQ_DECODE_PLAN");
     if (!e) return 0;
