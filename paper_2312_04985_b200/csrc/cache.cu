@@ -57,12 +57,14 @@ cache_append_kernel(const sparq_half* __restrict__ k_new, const sparq_half* __re
     }
 }
 
-// grid (ceil(S_max/64), B*Hkv), 256 threads: Kt[:, t0:t0+64] = K[t0:t0+64, :]^T for t < n.
+// one CTA of 256 threads per (KV head, block of 64 positions), one-dimensional grid:
+// Kt[:, t0:t0+64] = K[t0:t0+64, :]^T for t < n.
 __global__ void __launch_bounds__(256)
 cache_transpose_kernel(const sparq_half* __restrict__ K, sparq_half* __restrict__ Kt,
                        const int32_t* __restrict__ seq_lens, int Hkv, int S_max) {
     __shared__ uint16_t tile[64][D + 2];
-    const int bh = blockIdx.y, t0 = blockIdx.x * 64, tid = threadIdx.x;
+    const unsigned tblocks = (unsigned)(S_max + 63) / 64u;
+    const int bh = (int)(blockIdx.x / tblocks), t0 = (int)(blockIdx.x % tblocks) * 64, tid = threadIdx.x;
     const int n = min(seq_lens[bh / Hkv], S_max);
     if (t0 >= n) return;
     const size_t head = (size_t)bh * S_max * D;
@@ -105,8 +107,8 @@ cache_vsum_kernel(const sparq_half* __restrict__ V, const int32_t* __restrict__ 
 cudaError_t launch_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens, sparq_half* Kt,
                                float* vsum, sparq_half* vbar, int B, int Hkv, int S_max, int32_t* status,
                                cudaStream_t st) {
-    dim3 grid((S_max + 63) / 64, B * Hkv);
-    cache_transpose_kernel<<<grid, 256, 0, st>>>(K, Kt, seq_lens, Hkv, S_max);
+    const unsigned tblocks = (unsigned)(S_max + 63) / 64u;
+    cache_transpose_kernel<<<tblocks * (unsigned)(B * Hkv), 256, 0, st>>>(K, Kt, seq_lens, Hkv, S_max);
     cache_vsum_kernel<<<B * Hkv, 1024, 0, st>>>(V, seq_lens, vsum, vbar, Hkv, S_max, status);
     return cudaGetLastError();
 }

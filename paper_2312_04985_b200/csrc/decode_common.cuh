@@ -675,7 +675,8 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     // alpha = approximate-score mass of the selected set (Step 3)
     float apart = 0.f;
     for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[sc.i2[j]]) - vmax) * c1);
-    const float alpha = group_sum<G>(apart, sc.red, gtid) / Z;
+    // (numerator and denominator are fp32 sums taken in different orders: keep the mass a probability)
+    const float alpha = fminf(group_sum<G>(apart, sc.red, gtid) / Z, 1.0f);
     POST_CLK(4);
 
     // -------------------------------------------------------------- a5: gather k rows of K and V

@@ -1,5 +1,5 @@
 // dense_decode: dense single-token decode attention, Eq. (2), the comparison kernel for the
-// speed-up figure.  grid (splits, Hkv, B): a CTA covers one slice of the sequence of one KV head
+// speed-up figure.  One CTA per (split, KV head, batch): a CTA covers one slice of the sequence of one KV head
 // for all (up to 8 at a time) query heads of its group, so K and V are read once per KV head;
 // half-warp per cache row, 128-bit loads, online softmax in fp32.  With more than one split the
 // per-split softmax states go through a scratch buffer and a small merge kernel.
@@ -22,7 +22,7 @@ std::mutex g_dense_scratch_mutex;
 constexpr int NT = 256;             // threads per CTA
 constexpr int NHW = NT / 16;        // half-warps per CTA (one K/V row each)
 
-// grid (splits, Hkv, B).  A CTA covers positions [split*chunk, (split+1)*chunk) of one KV head
+// One CTA per (split, KV head, batch).  A CTA covers positions [split*chunk, (split+1)*chunk) of one KV head
 // for all G query heads of the group; half-warp per cache row, online softmax in fp32.
 template <int G>
 __global__ void __launch_bounds__(NT)
@@ -32,7 +32,9 @@ dense_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                     sparq_half* __restrict__ out, float* __restrict__ ws, int32_t* status) {
     __shared__ float merge[NHW * (D + 2)];
     const int tid = threadIdx.x, hw = tid >> 4, l16 = tid & 15;
-    const int split = blockIdx.x, hkv = blockIdx.y, b = blockIdx.z;
+    // one-dimensional grid: split fastest, then KV head, then batch (no 65535 limit on the batch)
+    const int split = (int)(blockIdx.x % (unsigned)splits);
+    const int hkv = (int)((blockIdx.x / (unsigned)splits) % (unsigned)Hkv), b = (int)(blockIdx.x / ((unsigned)splits * (unsigned)Hkv));
     const int n = seq_lens[b];
     const int h0 = hkv * g_total + g_base;                    // first query head served here
     if (n < 1 || n > S_max) {
@@ -195,7 +197,7 @@ cudaError_t launch_dense_decode(const sparq_half* q, const sparq_half* K, const 
                                 cudaStream_t st) {
     const int splits = dense_splits(B, Hkv, S_max);
     const int g = Hq / Hkv;
-    dim3 grid(splits, Hkv, B);
+    const unsigned grid = (unsigned)splits * (unsigned)Hkv * (unsigned)B;
     // the group's query heads are served G at a time by one pass over K and V
     for (int g_base = 0; g_base < g;) {
         int left = g - g_base;

@@ -236,7 +236,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
 
 // ---------------------------------------------------------------------------------- split-S plan
 // For fewer (batch, head) units than SMs (batch-1 decode over a long cache) and for caches whose
-// keys do not fit the persistent kernel's shared memory: grid (splits, units), 128 threads, five
+// keys do not fit the persistent kernel's shared memory: one CTA per (unit, slice), 128 threads, five
 // CTAs per SM.  Every unit's sequence is cut into `splits` interleaved slices; each CTA repeats
 // a1 (cheap) and streams its slice of the r selected Kt rows with plain 128-bit loads (16 rows in
 // flight per thread).  The keys go to a scratch buffer in global memory; the histogram of their top
@@ -286,7 +286,8 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     static_assert(SPLIT_FBINS <= HIST_BINS, "the first-digit histogram aliases the select scratch's histogram");
     __shared__ SplitShared sh;
     HeadMeta& hm = sh.hm;
-    const int tid = threadIdx.x, p = blockIdx.x, bh = blockIdx.y;
+    // one-dimensional grid (no 65535 limit on the units): the slices of a unit are neighbours in launch order
+    const int tid = threadIdx.x, p = (int)(blockIdx.x % (unsigned)splits), bh = (int)(blockIdx.x / (unsigned)splits);
     const int b = bh / Hq, h = bh % Hq, hkv = h / (Hq / Hkv);
     const int n = seq_lens[b];
     const size_t kv_head = (size_t)b * Hkv + hkv;
@@ -559,7 +560,7 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
         e = cudaMemsetAsync(ws_count, 0, (size_t)units * sizeof(unsigned int), stream);
         if (e != cudaSuccess) return e;
     }
-    kernel<<<dim3(splits, units), FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
+    kernel<<<(unsigned)splits * (unsigned)units, FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
                                                      post_bm_words(S_max), out, idx_r, idx_k, alpha, status,
                                                      ws_keys, ws_part, ws_hist, ws_count);
     return cudaGetLastError();

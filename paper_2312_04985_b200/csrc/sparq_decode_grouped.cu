@@ -90,7 +90,8 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     __shared__ GroupShared sh;
     HeadMeta& hm = sh.hm;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bk = blockIdx.y, b = bk / Hkv, p = blockIdx.x;              // (batch, KV head), slice
+    // one-dimensional grid: (batch, KV head) and slice, the slices of a group neighbours in launch order
+    const int bk = (int)(blockIdx.x / (unsigned)slices), b = bk / Hkv, p = (int)(blockIdx.x % (unsigned)slices);
     const int Hq = Hkv * G;
     const size_t q_row0 = ((size_t)b * Hq + (size_t)(bk % Hkv) * G) * D;  // first query head of the group
     const int n = seq_lens[b];
@@ -354,7 +355,7 @@ cudaError_t launch_g(const sparq_half* q, const sparq_half* K, const sparq_half*
         e = cudaMemsetAsync(ws_count, 0, (size_t)groups * sizeof(unsigned int), stream);
         if (e != cudaSuccess) return e;
     }
-    sparq_grouped_kernel<G><<<dim3(slices, groups), NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hkv, S_max, r, k, realloc,
+    sparq_grouped_kernel<G><<<(unsigned)slices * (unsigned)groups, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hkv, S_max, r, k, realloc,
                                                                       grouped_bm_words(S_max), slices, out, idx_r, idx_k,
                                                                       alpha, status, ws, ws_part, ws_count);
     return cudaGetLastError();

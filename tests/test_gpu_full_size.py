@@ -26,6 +26,10 @@ class FullCache:
         self.vbar = torch.zeros(B, Hkv, d, dtype=torch.float16, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         sparq.sparq_cache_build(self.K, self.V, self.seq, self.Kt, self.vsum, self.vbar, self.status)
+        # the workspace bench.py passes: the persistent kernel's unit counter on c2, the split plan's scratch on c3/c4
+        nbytes = sparq.sparq_workspace_bytes(B, case.Hq, Hkv, d, S_max, case.r, case.k)
+        assert nbytes > 0
+        self.ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
 
     def step(self, i):
         c = self.c
@@ -36,7 +40,7 @@ class FullCache:
         i2 = torch.empty(c.B, c.Hq, c.k, dtype=torch.int32, device=self.K.device)
         al = torch.empty(c.B, c.Hq, dtype=torch.float32, device=self.K.device)
         sparq.sparq_decode(c.q_steps[i], self.K, self.Kt, self.V, self.vbar, self.seq, c.r, c.k, out, idx_r=i1, idx_k=i2,
-                           alpha=al, status=self.status)
+                           alpha=al, workspace=self.ws, status=self.status)
         torch.cuda.synchronize()
         return out, i1, i2, al
 
