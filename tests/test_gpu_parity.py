@@ -129,6 +129,18 @@ def test_cache_longer_than_shared_memory_goes_through_the_workspace():
     assert e.value.code == sparq.ERR_TOO_LONG
 
 
+@pytest.mark.parametrize("plan", [None, "split"])
+def test_more_units_than_a_grid_dimension(plan):
+    """67,200 (batch, head) units: more than the 65,535 a second grid dimension could index; both the
+    persistent kernel (units drawn from the counter) and the split plan's one-dimensional grid."""
+    c = synth.make_case("c2", device="cuda", B=2100, Hq=32, Hkv=1, S=2048, r=16, k=32, ragged=(1200, 2047))
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    with H.decode_plan(plan):
+        waived, total = H.run_case_all_heads(c, "67200 units")
+    assert total == 67200 and waived <= 70
+
+
 def test_dense_decode_on_workloads():
     for name, kw in (("c1", {}), ("c3", dict(B=2, S=5000, backend="numpy")),
                      ("c4", dict(B=3, n_steps=1, ragged=(700, 2500), backend="numpy"))):
