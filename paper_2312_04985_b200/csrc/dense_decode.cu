@@ -49,15 +49,17 @@ dense_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     const int t_begin = split * chunk, t_end = min(n, t_begin + chunk);
 
     const float qscale = rsqrtf((float)D) * LOG2E;
-    float qs[G][8], acc[G][8], m[G], l[G];
+    // this lane's 8 query components per head, as stored (fp16): q . k is a chain of mixed-precision
+    // FMAs on exact fp16 x fp16 products, scaled once at the end
+    uint32_t qw[G][4];
+    float acc[G][8], m[G], l[G];
 #pragma unroll
     for (int gi = 0; gi < G; ++gi) {
         m[gi] = -CUDART_INF_F; l[gi] = 0.f;
+        const uint4 q8 = *reinterpret_cast<const uint4*>(q + ((size_t)b * Hq + h0 + gi) * D + l16 * 8);
+        qw[gi][0] = q8.x; qw[gi][1] = q8.y; qw[gi][2] = q8.z; qw[gi][3] = q8.w;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            qs[gi][e] = __half2float(__ushort_as_half(q[((size_t)b * Hq + h0 + gi) * D + l16 * 8 + e])) * qscale;
-            acc[gi][e] = 0.f;
-        }
+        for (int e = 0; e < 8; ++e) acc[gi][e] = 0.f;
     }
     const size_t kv_head = (size_t)b * Hkv + hkv;
     const uint4* Kh = reinterpret_cast<const uint4*>(K + kv_head * (size_t)S_max * D);
@@ -73,31 +75,44 @@ dense_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
             vv[u] = ld_stream(Vh + (size_t)t * (D / 8) + l16);
         }
 #pragma unroll
-        for (int u = 0; u < RG; ++u) {
-            const __half2* kh = reinterpret_cast<const __half2*>(&kv[u]);
-            const __half2* vh = reinterpret_cast<const __half2*>(&vv[u]);
-            float kf[8], vf[8];
+        for (int gi = 0; gi < G; ++gi) {
+            // the RG rows' logits for this head, then ONE rescale of the running state per batch of rows
+            float z[RG], bmax = -CUDART_INF_F;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float2 f = __half22float2(kh[e]); kf[2 * e] = f.x; kf[2 * e + 1] = f.y;
-                float2 w = __half22float2(vh[e]); vf[2 * e] = w.x; vf[2 * e + 1] = w.y;
-            }
-            const bool valid = t0 + u * NHW < t_end;          // uniform within the half-warp
+            for (int u = 0; u < RG; ++u) {
+                const uint32_t kw[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+                float za = 0.f, zb = 0.f;
 #pragma unroll
-            for (int gi = 0; gi < G; ++gi) {
-                float z = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) z = fmaf(kf[e], qs[gi][e], z);
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
-                if (valid) {
-                    float mn = fmaxf(m[gi], z);
-                    float sc = exp2f(m[gi] - mn), p = exp2f(z - mn);
-                    l[gi] = l[gi] * sc + p;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[gi][e] = fmaf(p, vf[e], acc[gi][e] * sc);
-                    m[gi] = mn;
+                for (int e = 0; e < 4; ++e) {
+                    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(za) : "h"((uint16_t)(kw[e] & 0xffffu)), "h"((uint16_t)(qw[gi][e] & 0xffffu)));
+                    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(zb) : "h"((uint16_t)(kw[e] >> 16)), "h"((uint16_t)(qw[gi][e] >> 16)));
                 }
+                float zz = (za + zb) * qscale;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) zz += __shfl_xor_sync(FULL, zz, o);
+                z[u] = (t0 + u * NHW < t_end) ? zz : -CUDART_INF_F;        // uniform within the half-warp
+                bmax = fmaxf(bmax, z[u]);
+            }
+            const float mn = fmaxf(m[gi], bmax);
+            if (mn > -CUDART_INF_F) {
+                const float sc = exp2f(m[gi] - mn);
+                float lsum = l[gi] * sc;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[gi][e] *= sc;
+#pragma unroll
+                for (int u = 0; u < RG; ++u) {
+                    const float p = exp2f(z[u] - mn);
+                    lsum += p;
+                    const __half2* vh = reinterpret_cast<const __half2*>(&vv[u]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 w = __half22float2(vh[e]);
+                        acc[gi][2 * e] = fmaf(p, w.x, acc[gi][2 * e]);
+                        acc[gi][2 * e + 1] = fmaf(p, w.y, acc[gi][2 * e + 1]);
+                    }
+                }
+                l[gi] = lsum;
+                m[gi] = mn;
             }
         }
     }
