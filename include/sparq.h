@@ -71,9 +71,9 @@ enum {
     SPARQ_ERR_TOO_LONG = 5,      /* S_max exceeds sparq_max_seq_len() (or, with a workspace,
                                     SPARQ_S_MAX_WORKSPACE)                                      */
     SPARQ_ERR_CUDA = 6,          /* the CUDA runtime refused a launch or a copy                  */
-    SPARQ_ERR_ALIGNMENT = 8,     /* a tensor or workspace pointer is not 16-byte aligned          */
     SPARQ_ERR_STATIC_SCRATCH = 7,/* the problem needs more scratch than the library's fixed
                                     SPARQ_STATIC_SCRATCH_BYTES: use the call that takes a workspace */
+    SPARQ_ERR_ALIGNMENT = 8,     /* a tensor or workspace pointer is not 16-byte aligned         */
     SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */
     SPARQ_DEV_CACHE_FULL = 17,   /* device: append with seq_lens[b] == S_max; nothing written    */
     SPARQ_DEV_TIMEOUT = 18       /* device: an asynchronous copy did not land within the bounded wait;
@@ -93,7 +93,8 @@ int sparq_max_seq_len(void);
  * sparq_cache_build -- derive the SparQ-specific cache state from a prefilled K, V:
  * Kt[b,h,:,t] = K[b,h,t,:] for t < seq_lens[b] (Section 6, "store K twice"), the fp32
  * running sum vsum = sum_{t<n} V[b,h,t,:] and vbar = fp16(vsum / n) (Section 3, v_bar).
- * Positions t >= seq_lens[b] of Kt are left untouched.  seq_lens[b] == 0 gives vsum = vbar = 0.
+ * Kt gets zeros from position seq_lens[b] to the end of its 16-byte vector (the layout's
+ * invariant); positions beyond that are left untouched.  seq_lens[b] == 0 gives vsum = vbar = 0.
  */
 int sparq_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
                       sparq_half* Kt, float* vsum, sparq_half* vbar,
