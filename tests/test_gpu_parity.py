@@ -99,6 +99,17 @@ def test_more_units_than_sms_all_heads():
     assert total == 672 and waived <= 3
 
 
+def test_persistent_kernel_with_three_key_buffers():
+    """A cache too long for the persistent kernel's four key buffers but short enough for three:
+    that instantiation walks several units per CTA, so its buffer slots wrap too."""
+    c = synth.make_case("c2", device="cuda", B=10, S=5120, ragged=(4700, 5119))       # 320 units
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    with H.decode_plan("pipe"):
+        waived, total = H.run_case_all_heads(c, "three key buffers")
+    assert total == 320 and waived <= 2
+
+
 def test_split_plan_unsliced_many_units():
     """The split plan with enough units to fill the GPU without slicing: every CTA streams a whole
     unit and goes straight on to the select and gather stages (no tickets, no histogram exchange)."""
