@@ -24,7 +24,9 @@ Readings taken where the paper is silent:
   * an all-zero query gives tau := 1 (all approximate logits are 0);
   * under grouped-query attention every query head selects for itself over the KV head
     ``h // g`` it shares (``sparq_decode``); the paper's own grouped variant, one selection
-    per KV head from sums over its query heads, is ``sparq_group_decode``.
+    per KV head from sums over its query heads, is ``sparq_group_decode``;
+  * the ablation settings (other temperatures, no reallocation) and the local window are
+    ``sparq_decode_opt``; their readings are stated above that function.
 
 Pins (tests/test_oracle_*.py): Figure "SparQ for a single attention head" worked numbers,
 closed forms of Eq. (9), reduction to Eq. (2) at r = d_h and k = S, brute force over all
@@ -369,6 +371,106 @@ def sparq_group_decode(q, K, V, seq_lens, r, k, v_bar=None, realloc=True):
             alpha[b, hkv * g:(hkv + 1) * g] = res["alpha"]
             gap_r[b, hkv] = res["gap_r"]
             gap_k[b, hkv] = res["gap_k"]
+    return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k)
+
+
+# --------------------------------------------------------------------------- ablation settings, local window
+# Section 5.3, "Approximate softmax temperature": besides Eq. (9) the paper evaluates tau = sqrt(d_h),
+# tau = sqrt(r), and the step without reallocation to the mean value.  Appendix, hyper-parameter
+# table: SparQ is listed with a "local window" l = k/4.
+# Readings:
+#   * the temperature only rescales the approximate logits, so i1 and i2 do not depend on it;
+#     alpha does;
+#   * "no reallocation" returns y3 of Eq. (8) itself.  In Eq. (10)'s notation that is alpha = 1
+#     (the limit tau -> 0, where s_hat becomes one-hot and its mass on the top-k set is 1); the
+#     ablation paragraph labels the same setting by the reallocated share being 0.  alpha is still
+#     reported as Eq. (10) defines it;
+#   * the local window's mechanism is not described anywhere for SparQ.  Taken here (a guess, by
+#     analogy with the window of the eviction baseline the paper compares with): the l most
+#     recent positions are always part of i2, inside the budget of k, and the other k - l places
+#     go to the largest approximate scores among the older positions; alpha sums s_hat over all
+#     of i2.  l is clipped to min(k, n).
+TAU_MODES = ("l1", "sqrt_d", "sqrt_r")
+
+
+def temperature_variant(q: np.ndarray, i1: np.ndarray, mode: str) -> float:
+    """tau of the approximate softmax: Eq. (9) ("l1"), sqrt(d_h) or sqrt(r)."""
+    if mode == "l1":
+        return temperature(q, i1)
+    if mode == "sqrt_d":
+        return math.sqrt(np.asarray(q).shape[0])
+    if mode == "sqrt_r":
+        return math.sqrt(len(i1))
+    raise ValueError("tau mode must be one of %s" % (TAU_MODES,))
+
+
+def top_k_window(l_hat: np.ndarray, k: int, window: int):
+    """Step 2 with a local window: i2 = the l most recent positions and the k_eff - l positions
+    with the largest approximate logit among the n - l older ones (ties to the smaller position),
+    k_eff = min(k, n), l = min(window, k_eff); alpha = sum of s_hat over i2.  ``gap`` is the
+    relative gap at the boundary of the ranked part (inf when nothing is ranked or rejected)."""
+    l_hat = np.asarray(l_hat, dtype=F64)
+    n = l_hat.shape[0]
+    if window < 0:
+        raise ValueError("window must be >= 0")
+    k_eff = max(0, min(int(k), n))
+    if k_eff == 0:
+        return np.zeros(0, dtype=np.int64), 0.0, math.inf
+    l = min(int(window), k_eff)
+    n_old, k_old = n - l, k_eff - l
+    order = _desc_order(l_hat[:n_old])
+    sel = np.concatenate([order[:k_old], np.arange(n_old, n)])
+    s_hat = softmax(l_hat)
+    alpha = float(np.sum(s_hat[sel]))
+    gap = math.inf if (k_old == 0 or k_old == n_old) else _rel_gap(l_hat[order[k_old - 1]], l_hat[order[k_old]])
+    return np.sort(sel).astype(np.int64), alpha, gap
+
+
+def sparq_head_opt(q, K, V, v_bar, n, r, k, tau_mode="l1", realloc=True, window=0):
+    """The SparQ step for one head with the ablation settings and the local window above;
+    ``tau_mode="l1", realloc=True, window=0`` is :func:`sparq_head`."""
+    if n < 1:
+        raise ValueError("sequence length must be >= 1")
+    q = np.asarray(q, dtype=F64)
+    i1, gap_r = top_r(q, r)
+    tau = temperature_variant(q, i1, tau_mode)
+    l_hat = (np.asarray(K[:n][:, i1], dtype=F64) @ q[i1]) / tau
+    i2, alpha, gap_k = top_k_window(l_hat, k, window)
+    if len(i2) == 0:
+        out = np.asarray(v_bar, dtype=F64).copy()
+    else:
+        y3 = attend(q, K, V, i2)
+        out = combine(alpha, y3, v_bar) if realloc else y3
+    return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k, tau=tau, l_hat=l_hat)
+
+
+def sparq_decode_opt(q, K, V, seq_lens, r, k, tau_mode="l1", realloc=True, window=0, v_bar=None):
+    """:func:`sparq_decode` with the settings of :func:`sparq_head_opt` (same shapes, same
+    per-query-head selection, same result dictionary)."""
+    q = np.asarray(q)
+    B, Hq, d = q.shape
+    Hkv = K.shape[1]
+    g = Hq // Hkv
+    out = np.zeros((B, Hq, d), dtype=F64)
+    i1 = np.zeros((B, Hq, r), dtype=np.int64)
+    i2 = -np.ones((B, Hq, k), dtype=np.int64)
+    alpha = np.zeros((B, Hq), dtype=F64)
+    gap_r = np.zeros((B, Hq), dtype=F64)
+    gap_k = np.zeros((B, Hq), dtype=F64)
+    for b in range(B):
+        n = int(seq_lens[b])
+        for hkv in range(Hkv):
+            Kh = np.asarray(K[b, hkv, :n], dtype=F64)
+            Vh = np.asarray(V[b, hkv, :n], dtype=F64)
+            vb = mean_value(Vh, n) if v_bar is None else np.asarray(v_bar[b, hkv], dtype=F64)
+            for h in range(hkv * g, (hkv + 1) * g):
+                res = sparq_head_opt(np.asarray(q[b, h], dtype=F64), Kh, Vh, vb, n, r, k, tau_mode, realloc, window)
+                out[b, h] = res["out"]
+                i1[b, h] = res["i1"]
+                i2[b, h, : len(res["i2"])] = res["i2"]
+                alpha[b, h] = res["alpha"]
+                gap_r[b, h] = res["gap_r"]
+                gap_k[b, h] = res["gap_k"]
     return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k)
 
 
