@@ -74,6 +74,7 @@ enum {
     SPARQ_ERR_STATIC_SCRATCH = 7,/* the problem needs more scratch than the library's fixed
                                     SPARQ_STATIC_SCRATCH_BYTES: use the call that takes a workspace */
     SPARQ_ERR_ALIGNMENT = 8,     /* a tensor or workspace pointer is not 16-byte aligned         */
+    SPARQ_ERR_BAD_OPTION = 9,    /* sparq_decode_opt: unknown temperature or window out of range */
     SPARQ_DEV_BAD_SEQ_LEN = 16,  /* device: seq_lens[b] < 1 or > S_max; that out row is zero     */
     SPARQ_DEV_CACHE_FULL = 17,   /* device: append with seq_lens[b] == S_max; nothing written    */
     SPARQ_DEV_TIMEOUT = 18       /* device: an asynchronous copy did not land within the bounded wait;
@@ -141,6 +142,32 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
                  sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                  void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k);
+
+/*
+ * sparq_decode_opt -- sparq_decode with the settings the paper varies around the algorithm
+ * (Section 5.3, "Approximate softmax temperature"; appendix, hyper-parameter table).  Same
+ * tensors, outputs, workspace (sparq_workspace_bytes()) and kernels as sparq_decode, which is
+ * this call with tau_mode = SPARQ_TAU_L1, realloc = 1, window = 0.
+ *   tau_mode  temperature of the approximate softmax of Eq. (7): SPARQ_TAU_L1 = Eq. (9),
+ *             SPARQ_TAU_SQRT_D = sqrt(d), SPARQ_TAU_SQRT_R = sqrt(r).  i1 and i2 do not depend
+ *             on it (the order of the approximate scores is the same); alpha does.
+ *   realloc   0: Step 3 is left out, out = y3 of Eq. (8) (the ablation's setting without
+ *             reallocation to the mean value); alpha is still written as Eq. (10) defines it.
+ *   window    local window l, 0 <= l <= SPARQ_K_MAX: the l_eff = min(l, k_eff) most recent
+ *             positions n - l_eff .. n - 1 always belong to i2, inside the budget of k, and the
+ *             other k_eff - l_eff places go to the largest approximate scores among the older
+ *             positions (ties to the smaller position); alpha sums s_hat over all of i2.  The
+ *             paper lists l = k/4 among SparQ's settings without describing the mechanism: this
+ *             is this library's reading of it.
+ * Returns SPARQ_ERR_BAD_OPTION for another tau_mode or window, before anything is launched.
+ */
+enum { SPARQ_TAU_L1 = 0, SPARQ_TAU_SQRT_D = 1, SPARQ_TAU_SQRT_R = 2 };
+int sparq_decode_opt(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                     const sparq_half* vbar, const int32_t* seq_lens,
+                     int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                     int tau_mode, int realloc, int window,
+                     sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                     void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
  * dense_decode -- dense decode attention, Eq. (2), over the n = seq_lens[b] valid positions:

@@ -65,6 +65,7 @@ const char* sparq_status_string(int code) {
         case SPARQ_ERR_CUDA: return "SPARQ_ERR_CUDA";
         case SPARQ_ERR_STATIC_SCRATCH: return "SPARQ_ERR_STATIC_SCRATCH";
         case SPARQ_ERR_ALIGNMENT: return "SPARQ_ERR_ALIGNMENT";
+        case SPARQ_ERR_BAD_OPTION: return "SPARQ_ERR_BAD_OPTION";
         case SPARQ_DEV_BAD_SEQ_LEN: return "SPARQ_DEV_BAD_SEQ_LEN";
         case SPARQ_DEV_CACHE_FULL: return "SPARQ_DEV_CACHE_FULL";
         case SPARQ_DEV_TIMEOUT: return "SPARQ_DEV_TIMEOUT";
@@ -119,11 +120,12 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     return 0;
 }
 
-int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
-                 const sparq_half* vbar, const int32_t* seq_lens,
-                 int B, int Hq, int Hkv, int d, int S_max, int r, int k,
-                 sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+// sparq_decode and sparq_decode_opt: one plan selection, the settings travel as one packed word
+static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                       const sparq_half* vbar, const int32_t* seq_lens,
+                       int B, int Hq, int Hkv, int d, int S_max, int r, int k, uint32_t opts,
+                       sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                       void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
     if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
@@ -138,7 +140,7 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
     const bool split_pays = split_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin()));
     if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
-        return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
+        return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
                                             alpha, status, splits, workspace, false, (cudaStream_t)stream));
     if (too_long) return SPARQ_ERR_TOO_LONG;                 // a plan without scratch was forced
     const bool fits = pipe_fits(S_max, device_smem_optin());
@@ -147,11 +149,32 @@ int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt,
         // with a workspace the persistent CTAs draw their units from a counter instead of a fixed share
         unsigned int* counter = (workspace && workspace_bytes >= SPARQ_PIPE_WORKSPACE_BYTES && B * Hq > n_sm)
                                     ? static_cast<unsigned int*>(workspace) : nullptr;
-        return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k,
+        return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
                                            alpha, status, n_sm, counter, (cudaStream_t)stream));
     }
-    return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
+    return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha,
                                   status, (cudaStream_t)stream));
+}
+
+int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                 const sparq_half* vbar, const int32_t* seq_lens,
+                 int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                 sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                 void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    return decode_with(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, 0u, out, idx_r, idx_k, alpha, workspace,
+                       workspace_bytes, status, stream);
+}
+
+int sparq_decode_opt(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                     const sparq_half* vbar, const int32_t* seq_lens,
+                     int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                     int tau_mode, int realloc, int window,
+                     sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                     void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (tau_mode < SPARQ_TAU_L1 || tau_mode > SPARQ_TAU_SQRT_R || window < 0 || window > SPARQ_K_MAX)
+        return SPARQ_ERR_BAD_OPTION;
+    return decode_with(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, pack_opts(tau_mode, realloc != 0, window),
+                       out, idx_r, idx_k, alpha, workspace, workspace_bytes, status, stream);
 }
 
 static int one_k_splits(int units, int S_max) {
@@ -175,7 +198,7 @@ int sparq_decode_1xk(const sparq_half* q, const sparq_half* K, const sparq_half*
     if (misaligned(q, K, V, vbar, out, workspace)) return SPARQ_ERR_ALIGNMENT;
     const int splits = one_k_splits(B * Hq, S_max);
     if (!workspace || workspace_bytes < split_scratch_bytes(B * Hq, S_max, splits)) return SPARQ_ERR_WORKSPACE;
-    return rc(launch_sparq_decode_split(q, K, nullptr, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, out, idx_r, idx_k, alpha,
+    return rc(launch_sparq_decode_split(q, K, nullptr, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, 0u, out, idx_r, idx_k, alpha,
                                         status, splits, workspace, true, (cudaStream_t)stream));
 }
 

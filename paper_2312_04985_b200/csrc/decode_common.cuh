@@ -40,7 +40,27 @@ struct alignas(16) HeadMeta {
     uint16_t qh[D + 8];           // selected components' fp16 bits in i1 order, zero padded
     int32_t bh, n, k_eff, valid;
     float inv_tau, l1_sel;
+    int32_t n_sel, k_sel;         // Step 2 ranks positions [0, n_sel) for k_sel places; [n_sel, n) is the local window
 };
+
+// Settings of a decode call packed into one word (0 = the paper's algorithm as Section 4 states it):
+// bits 0-1 the approximate softmax's temperature (0: Eq. (9), 1: sqrt(d_h), 2: sqrt(r); Section 5.3),
+// bit 2 set: Step 3 left out (the output is Eq. (8)'s y3), bits 16-31: local window l.  Packed on the
+// host by pack_opts() (kernels.h).
+__device__ __forceinline__ bool opt_realloc(uint32_t opts) { return (opts & 4u) == 0u; }
+// 1 / tau.  Eq. (9) with tau := 1 where it is 0/0 (no weight on the kept components: every approximate logit is 0).
+__device__ __forceinline__ float opt_inv_tau(uint32_t opts, float l1_all, float l1_sel, int r) {
+    const uint32_t mode = opts & 3u;
+    if (mode == 1u) return rsqrtf((float)D);
+    if (mode == 2u) return rsqrtf((float)r);
+    return (l1_all > 0.f && l1_sel > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
+}
+// The l = min(window, k_eff) most recent positions are selected outright; the other places are ranked.
+__device__ __forceinline__ void opt_set_window(HeadMeta& hm, int n, int k_eff, uint32_t opts) {
+    const int l = min((int)(opts >> 16), k_eff);
+    hm.n_sel = n - l;
+    hm.k_sel = k_eff - l;
+}
 
 // Shared-memory scratch of one post phase.
 struct PostScratch {
@@ -299,7 +319,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
                                                        float kabs, const PostScratch& sc, int r, int S_max,
                                                        const sparq_half* __restrict__ Kt_head, int t_stride = 1) {
     const int lane = gtid & 31, warp = gtid >> 5;
-    const int n = hm.n, k_eff = hm.k_eff;
+    const int n = hm.n_sel, k_eff = hm.k_sel;                // the ranked positions and places (all of them without a window)
     const float inv_tau = hm.inv_tau;
     const float vmax = unkey32(kmax);
     const float twoB = two_b(r, hm.l1_sel, kabs);
@@ -338,16 +358,16 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
     // -------------------------------------------------------------- a3 + bitmap of the selection
     // Softmax denominator, the speculative selection key >= edge as a bitmap, and the positions
     // whose key lies within 2B of the edge (counted on each side, listed while the list has room).
-    const int nwords = (n + 31) >> 5;
+    const int nwords = (hm.n + 31) >> 5;                     // the denominator runs over the window too
     const float c1 = inv_tau * LOG2E;
     if (gtid < 4) sc.band[gtid] = 0;
     G::sync();
     float zpart = 0.f;
     for (int wi = warp; wi < nwords; wi += G::NW) {
         const int t = (wi << 5) + lane;
+        const uint32_t u = t < hm.n ? keys[t] : 0u;
+        zpart += t < hm.n ? ex2((unkey32(u) - vmax) * c1) : 0.f;
         const bool valid = t < n;
-        const uint32_t u = valid ? keys[t] : 0u;
-        zpart += valid ? ex2((unkey32(u) - vmax) * c1) : 0.f;
         const bool ge = valid && u >= edge;
         const unsigned g = __ballot_sync(FULL, ge);
         if (lane == 0) sc.bm_sel[wi] = g;
@@ -443,7 +463,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     constexpr int FSH_ = 32 - FB_, FBINS_ = 1 << FB_;         // first digit: the keys' top FB_ bits
     static_assert(FSH_ > 16 && FSH_ <= 24, "the bin's remaining bits resolve as 8 + 8 + (FSH_ - 16)");
     const int lane = gtid & 31, warp = gtid >> 5;
-    const int n = hm.n, k_eff = hm.k_eff;
+    const int n = hm.n_sel, k_eff = hm.k_sel;                // the ranked positions and places (all of them without a window)
     (void)kmax;
 
     POST_CLK_INIT();
@@ -617,6 +637,43 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     }
     POST_CLK(3);
     return true;
+}
+
+// Local window, before a select that starts from a first-digit histogram of all n keys: take the
+// window's keys out of it again (at most SPARQ_K_MAX of them).  Ends with a barrier.
+template <class G, int FB_ = FB>
+__device__ __forceinline__ void window_unhist(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t* hist1) {
+    for (int t = hm.n_sel + gtid; t < hm.n; t += G::NT) atomicSub(&hist1[keys[t] >> (32 - FB_)], 1u);
+    G::sync();
+}
+
+// Local window, after the select: positions [n_sel, n) join the selection.  The select wrote the
+// bitmap words that hold ranked positions; the words above them are set here.  Ends with a barrier.
+template <class G>
+__device__ __forceinline__ void window_mark(int gtid, const HeadMeta& hm, const PostScratch& sc) {
+    const int n_sel = hm.n_sel, n = hm.n;
+    const int ranked_words = (n_sel + 31) >> 5;
+    for (int wi = (n_sel >> 5) + gtid; wi <= ((n - 1) >> 5); wi += G::NT) {
+        const int lo = max(n_sel - (wi << 5), 0), hi = min(n - (wi << 5), 32);       // bits [lo, hi) of this word
+        const uint32_t mask = (hi == 32 ? ~0u : (1u << hi) - 1u) & ~((1u << lo) - 1u);
+        sc.bm_sel[wi] = (wi < ranked_words ? sc.bm_sel[wi] : 0u) | mask;
+    }
+    G::sync();
+}
+
+// Local window as large as the budget (k_sel = 0): nothing is ranked.  Clears the bitmap words of the
+// older positions; Z = the softmax denominator relative to the largest key, from the keys.
+template <class G>
+__device__ __forceinline__ SelectResult select_nothing(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+                                                       const PostScratch& sc) {
+    const float vmax = unkey32(kmax), c1 = hm.inv_tau * LOG2E;
+    for (int wi = gtid; wi < ((hm.n_sel + 31) >> 5); wi += G::NT) sc.bm_sel[wi] = 0u;
+    float zpart = 0.f;
+    for (int t = gtid; t < hm.n; t += G::NT) zpart += ex2((unkey32(keys[t]) - vmax) * c1);
+    SelectResult res;
+    res.Z = group_sum<G>(zpart, sc.red, gtid);               // its barriers publish the bitmap
+    res.need_tie = 0;
+    return res;
 }
 
 // Stages a5 and a6 for one unit from a finished selection: ascending index list from the bitmap(s),

@@ -8,13 +8,20 @@
 
 namespace sparq {
 
+// `opts` of the decode launchers: the call's settings in one word (0 = Eq. (9) temperature, Step 3
+// applied, no local window).  Bits 0-1: temperature (SPARQ_TAU_*), bit 2: Step 3 left out,
+// bits 16-31: local window.
+inline uint32_t pack_opts(int tau_mode, int realloc, int window) {
+    return (uint32_t)tau_mode | (realloc ? 0u : 4u) | ((uint32_t)window << 16);
+}
+
 // sparq_decode.cu
 size_t decode_static_smem();
 size_t decode_dynamic_smem(int S_max);
 int decode_max_positions();
 cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                 const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                 int32_t* status, cudaStream_t stream);
 
 // split-S plan (sparq_decode.cu): one CTA per (slice, unit) with the keys in a scratch buffer, for
@@ -23,7 +30,7 @@ int split_count(int units, int S_max, int n_sm);
 size_t split_scratch_bytes(int units, int S_max, int splits);
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                       const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                      int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                       int32_t* status, int splits, void* scratch, bool one_k, cudaStream_t stream);
 
 // sparq_decode_pipe.cu: persistent warp-specialised variant for S_max small enough that three key
@@ -31,7 +38,7 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
 bool pipe_fits(int S_max, int smem_optin);
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                     int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                     int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                      int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream);
 
 // sparq_decode_grouped.cu: group-shared selection (one CTA per KV head)

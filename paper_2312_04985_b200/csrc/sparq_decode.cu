@@ -54,7 +54,7 @@ __device__ unsigned long long g_phase_clocks[16];
 // red: 2*NW floats, cnt: 4 words.  Ends with a barrier.
 template <class G, int RB_>
 __device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restrict__ q_row, int r, HeadMeta& hm, float* red,
-                                            uint32_t* cnt) {
+                                            uint32_t* cnt, uint32_t opts) {
     const int lane = tid & 31, warp = tid >> 5;
     uint16_t hb = 0;
     float qf = 0.f, aq = 0.f;
@@ -92,7 +92,7 @@ __device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restric
     }
     const int r_pad = (r + RB_ - 1) / RB_ * RB_;
     if (tid >= r && tid < r_pad) hm.qh[tid] = 0;
-    if (tid == 0) { hm.inv_tau = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f; hm.l1_sel = l1_sel; }
+    if (tid == 0) { hm.inv_tau = opt_inv_tau(opts, l1_all, l1_sel, r); hm.l1_sel = l1_sel; }
     G::sync();
 }
 
@@ -112,7 +112,7 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
                     const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
                     int Hq, int Hkv, int S_max, int r, int k,
                     sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
-                    float* __restrict__ alpha_out, int32_t* status) {
+                    float* __restrict__ alpha_out, int32_t* status, uint32_t opts) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;                                       // a2: STAGES x [RB rows x CH positions] fp16
     uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);  // [n] approximate-score keys
@@ -139,9 +139,10 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
         for (int s = 0; s < STAGES; ++s) mbar_init(&sh.full[s], 1);
         mbar_init_fence();
         hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = 1;
+        opt_set_window(hm, n, k_eff, opts);
     }
 
-    top_r_block<CTA, RB>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.res);        // a1
+    top_r_block<CTA, RB>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.res, opts);  // a1
     const int r_pad = (r + RB - 1) / RB * RB;
     if (idx_r) for (int j = tid; j < r; j += NT) idx_r[(size_t)bh * r + j] = hm.i1[j];
 
@@ -228,9 +229,12 @@ sparq_decode_kernel(const sparq_half* __restrict__ q, const sparq_half* __restri
     PostScratch sc;
     carve_post_scratch(sc, ring, CTA::NHW, BM_WORDS);
     sc.i2 = sh.i2; sc.red = sh.red; sc.redu = sh.redu; sc.res = sh.res; sc.band = sh.band;
-    const SelectResult sel_res = select_generic<CTA>(tid, hm, keys, kmax, __uint_as_float(kabs_bits), sc, r, S_max, Kt_head);
+    const SelectResult sel_res = hm.k_sel == 0 ? select_nothing<CTA>(tid, hm, keys, kmax, sc)
+                                               : select_generic<CTA>(tid, hm, keys, kmax, __uint_as_float(kabs_bits), sc, r, S_max, Kt_head);
+    if (hm.n_sel != hm.n) window_mark<CTA>(tid, hm, sc);
     finish<CTA, 8>(tid, hm, keys, kmax, sel_res, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
-                   vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
+                   vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr,
+                   true, opt_realloc(opts));
     PHASE_MARK(2);
 }
 
@@ -279,7 +283,7 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
                    int Hq, int Hkv, int S_max, int r, int k, int splits, int bm_words,
                    sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
                    float* __restrict__ alpha_out, int32_t* status,
-                   uint32_t* ws_keys, uint32_t* ws_part, uint32_t* ws_hist, unsigned int* ws_count) {
+                   uint32_t* ws_keys, uint32_t* ws_part, uint32_t* ws_hist, unsigned int* ws_count, uint32_t opts) {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     // histogram of the keys' top bits; once the threshold bin is known the space becomes the select stage's list
     uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn_smem);
@@ -305,8 +309,8 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     const int k_eff = min(k, n);
     PHASE_INIT();
     for (int i = tid; i < SPLIT_FBINS / 4; i += FNT) reinterpret_cast<uint4*>(hist1)[i] = make_uint4(0, 0, 0, 0);
-    if (tid == 0) { hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; }
-    top_r_block<FCTA, 8>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.cnt);      // a1; its barriers also publish the cleared histogram
+    if (tid == 0) { hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; opt_set_window(hm, n, k_eff, opts); }
+    top_r_block<FCTA, 8>(tid, q + (size_t)bh * D, r, hm, sh.red, sh.cnt, opts);   // a1; its barriers also publish the cleared histogram
     if (p == 0 && idx_r) for (int j = tid; j < r; j += FNT) idx_r[(size_t)bh * r + j] = hm.i1[j];
     if (k_eff == 0) {                    // nothing to select: the output is the mean value vector
         if (p == 0) {
@@ -470,15 +474,23 @@ sparq_split_kernel(const sparq_half* __restrict__ q, const sparq_half* __restric
     // where the fp64 re-decision finds component c of position t: Kt[c * S_max + t], or K[t * d_h + c]
     const sparq_half* band_src = ONE_K ? K + kv_head * (size_t)S_max * D : Kt_head;
     const int c_stride = ONE_K ? 1 : S_max, t_stride = ONE_K ? D : 1;
-    if (!select_prefilled<FCTA, SPLIT_FB, true>(tid, hm, keys, kmax, kabs, Z, sc, hist1, r, c_stride, band_src, sel, t_stride)) {
+    const bool windowed = hm.n_sel != hm.n;                  // (uniform) a local window is reserved inside the budget
+    if (hm.k_sel == 0) {
+        sel = select_nothing<FCTA>(tid, hm, keys, kmax, sc);
+    } else {
+        if (windowed) window_unhist<FCTA, SPLIT_FB>(tid, hm, keys, hist1);
+        if (!select_prefilled<FCTA, SPLIT_FB, true>(tid, hm, keys, kmax, kabs, Z, sc, hist1, r, c_stride, band_src, sel, t_stride)) {
 #ifdef SPARQ_PHASE_CLOCKS
-        if (tid == 0) atomicAdd(&g_phase_clocks[7], 1ull);
+            if (tid == 0) atomicAdd(&g_phase_clocks[7], 1ull);
 #endif
-        sel = select_generic<FCTA>(tid, hm, keys, kmax, kabs, sc, r, c_stride, band_src, t_stride);
+            sel = select_generic<FCTA>(tid, hm, keys, kmax, kabs, sc, r, c_stride, band_src, t_stride);
+        }
     }
+    if (windowed) window_mark<FCTA>(tid, hm, sc);
     PHASE_MARK(2);
     finish<FCTA, 4>(tid, hm, keys, kmax, sel, sc, k, K + kv_head * (size_t)S_max * D, V + kv_head * (size_t)S_max * D,
-                    vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr);
+                    vbar + kv_head * D, out_row, idx_k ? idx_k + (size_t)bh * k : nullptr, alpha_out ? alpha_out + bh : nullptr,
+                    true, opt_realloc(opts));
     PHASE_MARK(3);
 }
 
@@ -512,13 +524,13 @@ int decode_max_positions() { return BM_WORDS * 32; }
 
 cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                 const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                 int32_t* status, cudaStream_t stream) {
     const size_t dyn = decode_dynamic_smem(S_max);
     cudaError_t e = cudaFuncSetAttribute(sparq_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     sparq_decode_kernel<<<B * Hq, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, out, idx_r,
-                                                            idx_k, alpha, status);
+                                                            idx_k, alpha, status, opts);
     return cudaGetLastError();
 }
 
@@ -540,7 +552,7 @@ size_t split_scratch_bytes(int units, int S_max, int splits) {
 
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                       const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                      int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                       int32_t* status, int splits, void* scratch, bool one_k, cudaStream_t stream) {
     const int units = B * Hq;
     uint32_t* ws_keys = static_cast<uint32_t*>(scratch);
@@ -562,7 +574,7 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
     }
     kernel<<<(unsigned)splits * (unsigned)units, FNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, splits,
                                                      post_bm_words(S_max), out, idx_r, idx_k, alpha, status,
-                                                     ws_keys, ws_part, ws_hist, ws_count);
+                                                     ws_keys, ws_part, ws_hist, ws_count, opts);
     return cudaGetLastError();
 }
 

@@ -155,7 +155,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         // (a head with no weight on the group's components has all-zero approximate logits: tau := 1)
         if (tid == 0) sh.inv_tau[h] = (l1_all > 0.f && l1_sel > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
     }
-    if (tid == 0) { hm.bh = bk; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; hm.l1_sel = 0.f; }
+    if (tid == 0) { hm.bh = bk; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; hm.l1_sel = 0.f; hm.n_sel = n; hm.k_sel = k_eff; }
     __syncthreads();
     if (p == 0 && idx_r) for (int j = tid; j < r; j += NT) idx_r[(size_t)bk * r + j] = hm.i1[j];
 

@@ -124,7 +124,7 @@ __device__ __forceinline__ int next_unit(const Args& a, int bh, int lane) {
     return u < a.n_units ? u : -1;
 }
 
-__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
+__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uint32_t opts) {
     const int lane = threadIdx.x & 31;
     int bh = (int)blockIdx.x < a.n_units ? (int)blockIdx.x : -1;
     uint2 qraw = make_uint2(0, 0);                           // components 4*lane .. 4*lane+3 of the unit's q
@@ -139,7 +139,7 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
         HeadMeta& hm = sh.meta[m];
         if (bh < 0) {                                        // no unit left: an end marker for one post group
             wait_or_abort<200>(&sh.meta_free[m], (((uint32_t)(j / NMETA)) & 1u) ^ 1u, sh, a.status);
-            if (lane == 0) { hm.bh = -1; hm.n = 0; hm.k_eff = 0; hm.valid = 0; }
+            if (lane == 0) { hm.bh = -1; hm.n = 0; hm.k_eff = 0; hm.valid = 0; hm.n_sel = 0; hm.k_sel = 0; }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.meta_full[m]);
             ++markers;
@@ -191,8 +191,9 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh) {
         for (int c = a.r + lane; c < r_pad; c += 32) hm.qh[c] = 0;
         if (lane == 0) {
             hm.bh = bh; hm.n = n; hm.k_eff = k_eff; hm.valid = valid;
-            hm.inv_tau = (l1_all > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
+            hm.inv_tau = opt_inv_tau(opts, l1_all, l1_sel, a.r);
             hm.l1_sel = l1_sel;
+            opt_set_window(hm, n, k_eff, opts);
         }
         __syncwarp();
         if (a.idx_r) for (int c = lane; c < a.r; c += 32) a.idx_r[(size_t)bh * a.r + c] = valid ? hm.i1[c] : -1;
@@ -345,7 +346,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 // ---------------------------------------------------------------------------------- post groups
 template <class PG, int NKB>
 __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, uint32_t* hist1_all,
-                                          unsigned char* scratch, int p) {
+                                          unsigned char* scratch, int p, const uint32_t opts) {
     const int gtid = threadIdx.x - LEAD - SNT - p * GNT;
     PostScratch sc;
     carve_post_scratch(sc, scratch, PG::NHW, a.S_cap / 32);
@@ -378,12 +379,21 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             const uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
             const sparq_half* Kt_head = a.Kt + kv_head * (size_t)D * a.S_max;
             SelectResult sel;
-            if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sh.zsum[kb], sc, hist1_all + kb * FBINS, a.r,
-                                      a.S_max, Kt_head, sel))
-                sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
+            const bool windowed = (opts >> 16) != 0u && hm.n_sel != hm.n;   // (uniform) a local window is reserved inside the budget
+            if (windowed && hm.k_sel == 0) {                 // the window takes the whole budget: nothing to rank
+                for (int i = gtid; i < FBINS; i += GNT) hist1_all[kb * FBINS + i] = 0;   // left clear for the buffer's next unit
+                sel = select_nothing<PG>(gtid, hm, keys, sh.kmax[kb], sc);
+            } else {
+                if (windowed) window_unhist<PG>(gtid, hm, keys, hist1_all + kb * FBINS);
+                if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sh.zsum[kb], sc, hist1_all + kb * FBINS, a.r,
+                                          a.S_max, Kt_head, sel))
+                    sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
+            }
+            if (windowed) window_mark<PG>(gtid, hm, sc);
             finish<PG, 4>(gtid, hm, keys, sh.kmax[kb], sel, sc, a.k, a.K + kv_head * (size_t)a.S_max * D,
                           a.V + kv_head * (size_t)a.S_max * D, a.vbar + kv_head * D, out_row,
-                          a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr);
+                          a.idx_k ? a.idx_k + (size_t)bh * a.k : nullptr, a.alpha ? a.alpha + bh : nullptr, true,
+                          opt_realloc(opts));
         }
         PG::sync();                                          // the group is done with the keys, the metadata, i2
         CLK_ADD(0, t_p, gtid == 0);
@@ -391,8 +401,11 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
     }
 }
 
-template <int NKB>
-__global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) {
+// OPT = false: the paper's algorithm as stated, the settings word known to be 0 at compile time (the
+// instantiation the plain decode call runs); OPT = true: settings taken from `opts_arg`.
+template <int NKB, bool OPT>
+__global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, const uint32_t opts_arg) {
+    const uint32_t opts = OPT ? opts_arg : 0u;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
     uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);
@@ -415,10 +428,10 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a) 
 #endif
     const int warp = threadIdx.x >> 5;
     if (warp < NPROD) producer_role(a, sh, ring, warp);
-    else if (warp == NPROD) a1_role(a, sh);
+    else if (warp == NPROD) a1_role(a, sh, opts);
     else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB>(a, sh, ring, keys_all, hist1_all);
-    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB>(a, sh, keys_all, hist1_all, scratch0, 0);
-    else post_role<PG1, NKB>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1);
+    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB>(a, sh, keys_all, hist1_all, scratch0, 0, opts);
+    else post_role<PG1, NKB>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1, opts);
 }
 
 size_t pipe_dynamic_smem(int S_cap, int NKB) {
@@ -459,7 +472,7 @@ bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_opt
 
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                     int r, int k, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                                     int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
                                      int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream) {
     Args a;
     a.q = q; a.K = K; a.Kt = Kt; a.V = V; a.vbar = vbar; a.seq_lens = seq_lens;
@@ -470,16 +483,16 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
     cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     const bool four = pipe_fits_nkb(S_max, smem_optin, 4);
     const size_t dyn = pipe_dynamic_smem(a.S_cap, four ? 4 : 3);
-    cudaError_t e = four ? cudaFuncSetAttribute(sparq_decode_pipe_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn)
-                         : cudaFuncSetAttribute(sparq_decode_pipe_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+    auto kernel = opts ? (four ? sparq_decode_pipe_kernel<4, true> : sparq_decode_pipe_kernel<3, true>)
+                       : (four ? sparq_decode_pipe_kernel<4, false> : sparq_decode_pipe_kernel<3, false>);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     const int grid = a.n_units < n_sm ? a.n_units : n_sm;
     if (unit_counter) {
         e = cudaMemsetAsync(unit_counter, 0, sizeof(unsigned int), stream);
         if (e != cudaSuccess) return e;
     }
-    if (four) sparq_decode_pipe_kernel<4><<<grid, NT, dyn, stream>>>(a);
-    else sparq_decode_pipe_kernel<3><<<grid, NT, dyn, stream>>>(a);
+    kernel<<<grid, NT, dyn, stream>>>(a, opts);
     return cudaGetLastError();
 }
 

@@ -20,6 +20,8 @@ from . import build as _build
 OK = 0
 ERR_NULL_POINTER, ERR_BAD_SHAPE, ERR_BAD_RK, ERR_WORKSPACE, ERR_TOO_LONG, ERR_CUDA, ERR_STATIC_SCRATCH = 1, 2, 3, 4, 5, 6, 7
 ERR_ALIGNMENT = 8
+ERR_BAD_OPTION = 9
+TAU_L1, TAU_SQRT_D, TAU_SQRT_R = 0, 1, 2
 STATIC_SCRATCH_BYTES = 8 << 20
 DEV_BAD_SEQ_LEN, DEV_CACHE_FULL, DEV_TIMEOUT = 16, 17, 18
 K_MAX = 1024
@@ -28,7 +30,7 @@ HEAD_DIM = 128
 EXPORTS = ("sparq_status_string", "sparq_max_seq_len", "sparq_cache_build", "sparq_cache_append", "sparq_decode",
            "sparq_workspace_bytes", "dense_decode", "dense_workspace_bytes", "dense_decode_static", "sparq_step_host",
            "sparq_step_host_staging_bytes", "sparq_decode_grouped", "sparq_grouped_workspace_bytes",
-           "sparq_decode_1xk", "sparq_1xk_workspace_bytes")
+           "sparq_decode_1xk", "sparq_1xk_workspace_bytes", "sparq_decode_opt")
 
 
 class SparqError(RuntimeError):
@@ -60,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.sparq_cache_append.argtypes = [vp] * 8 + [i] * 4 + [vp, vp]
         L.sparq_decode.restype = i
         L.sparq_decode.argtypes = [vp] * 6 + [i] * 7 + [vp] * 4 + [vp, sz, vp, vp]
+        L.sparq_decode_opt.restype = i
+        L.sparq_decode_opt.argtypes = [vp] * 6 + [i] * 10 + [vp] * 4 + [vp, sz, vp, vp]
         L.sparq_workspace_bytes.restype = sz
         L.sparq_workspace_bytes.argtypes = [i] * 7
         L.dense_decode.restype = i
@@ -159,6 +163,24 @@ def sparq_decode(q, K, Kt, V, vbar, seq_lens, r, k, out, idx_r=None, idx_k=None,
                                 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                 _dev(status, torch.int32, "status"), _stream(q))
     _check("sparq_decode", rc)
+    return out
+
+
+def sparq_decode_opt(q, K, Kt, V, vbar, seq_lens, r, k, out, tau_mode=TAU_L1, realloc=True, window=0, idx_r=None,
+                     idx_k=None, alpha=None, workspace=None, status=None):
+    B, Hq, d = q.shape
+    Hkv, S_max = K.shape[1], K.shape[2]
+    with torch.cuda.device(q.device):
+        rc = lib().sparq_decode_opt(_dev(q, torch.float16, "q"), _dev(K, torch.float16, "K"),
+                                    _dev(Kt, torch.float16, "Kt"), _dev(V, torch.float16, "V"),
+                                    _dev(vbar, torch.float16, "vbar"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                    B, Hq, Hkv, d, S_max, int(r), int(k), int(tau_mode), 1 if realloc else 0, int(window),
+                                    _dev(out, torch.float16, "out"), _dev(idx_r, torch.int32, "idx_r"),
+                                    _dev(idx_k, torch.int32, "idx_k"), _dev(alpha, torch.float32, "alpha"),
+                                    None if workspace is None else workspace.data_ptr(),
+                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _dev(status, torch.int32, "status"), _stream(q))
+    _check("sparq_decode_opt", rc)
     return out
 
 

@@ -36,7 +36,7 @@ def test_every_declared_function_is_exported(lib):
 def test_status_strings(lib):
     codes = {0: "SPARQ_OK", 1: "SPARQ_ERR_NULL_POINTER", 2: "SPARQ_ERR_BAD_SHAPE", 3: "SPARQ_ERR_BAD_RK",
              4: "SPARQ_ERR_WORKSPACE", 5: "SPARQ_ERR_TOO_LONG", 6: "SPARQ_ERR_CUDA", 7: "SPARQ_ERR_STATIC_SCRATCH",
-             8: "SPARQ_ERR_ALIGNMENT",
+             8: "SPARQ_ERR_ALIGNMENT", 9: "SPARQ_ERR_BAD_OPTION",
              16: "SPARQ_DEV_BAD_SEQ_LEN", 17: "SPARQ_DEV_CACHE_FULL", 18: "SPARQ_DEV_TIMEOUT"}
     for code, name in codes.items():
         assert sparq.status_string(code) == name
@@ -59,6 +59,13 @@ def test_host_visible_errors_need_no_device(lib):
     # r and k ranges
     for r, k in ((0, 1), (129, 1), (4, -1), (4, sparq.K_MAX + 1)):
         assert lib.sparq_decode(one, one, one, one, one, one, 1, 1, 1, 128, 8, r, k, one, n, n, n, n, 0, n, n) == sparq.ERR_BAD_RK
+    # settings of sparq_decode_opt: unknown temperature, window out of range; its other checks are sparq_decode's
+    opt = lambda tau, realloc, window, q=one, r=1: lib.sparq_decode_opt(
+        q, one, one, one, one, one, 1, 1, 1, 128, 8, r, 1, tau, realloc, window, one, n, n, n, n, 0, n, n)
+    for tau, window in ((3, 0), (-1, 0), (0, -1), (0, sparq.K_MAX + 1)):
+        assert opt(tau, 1, window) == sparq.ERR_BAD_OPTION
+    assert opt(2, 0, 5, q=n) == sparq.ERR_NULL_POINTER
+    assert opt(2, 0, 5, r=0) == sparq.ERR_BAD_RK
     # a tensor pointer that is not 16-byte aligned (the kernels would fault on it)
     odd = ctypes.c_void_p(24)
     assert lib.sparq_decode(one, one, odd, one, one, one, 1, 1, 1, 128, 8, 1, 1, one, n, n, n, n, 0, n, n) == sparq.ERR_ALIGNMENT
