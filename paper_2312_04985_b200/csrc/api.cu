@@ -218,7 +218,7 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
     if (g != 1 && g != 2 && g != 4 && g != 8) return SPARQ_ERR_BAD_SHAPE;
     if (r < 1 || r > d || k < 0 || k > SPARQ_K_MAX) return SPARQ_ERR_BAD_RK;
     if (misaligned(q, K, Kt, V, vbar, out, workspace)) return SPARQ_ERR_ALIGNMENT;
-    if (S_max > SPARQ_S_MAX_WORKSPACE || grouped_dynamic_smem(S_max) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
+    if (S_max > SPARQ_S_MAX_WORKSPACE || grouped_dynamic_smem(S_max, Hq / Hkv, k) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
     const int slices = grouped_slices(B * Hkv, S_max, device_sm_count());
     if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices)) return SPARQ_ERR_WORKSPACE;
     return rc(launch_sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, realloc, out, idx_r, idx_k,

@@ -676,27 +676,13 @@ __device__ __forceinline__ SelectResult select_nothing(int gtid, const HeadMeta&
     return res;
 }
 
-// Stages a5 and a6 for one unit from a finished selection: ascending index list from the bitmap(s),
-// alpha, gather of the selected K and V rows with online softmax, combine with v_bar.
-// RG: gathered K and V rows in flight per half-warp (register budget of the calling kernel).
-// realloc = false leaves Step 3 out (out = the restricted attention; alpha is still reported).
-// Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
-// group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
-template <class G, int RG>
-__device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, SelectResult sel,
-                                       const PostScratch& sc, int k, const sparq_half* __restrict__ K_head,
-                                       const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
-                                       sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
-                                       float* __restrict__ alpha_out, bool build_list = true, bool realloc = true) {
+// The ascending list sc.i2 of the k_eff selected positions from the selection bitmap (plus, in the
+// degenerate path, the first need_tie positions of the tie bitmap).  Ends with a barrier.
+template <class G>
+__device__ __forceinline__ void build_index_list(int gtid, const HeadMeta& hm, SelectResult sel, const PostScratch& sc) {
     const int n = hm.n, k_eff = hm.k_eff;
-    const int nwords = build_list ? (n + 31) >> 5 : 0;       // (a caller that kept sc.i2 from an earlier call skips the rebuild)
-    const float vmax = unkey32(kmax);
-    const float c1 = hm.inv_tau * LOG2E;
-    const float Z = sel.Z;
+    const int nwords = (n + 31) >> 5;
     const uint32_t need_tie = sel.need_tie;
-    POST_CLK_INIT();
-
-    // ascending list of selected positions from the bitmap(s)
     uint32_t carry_tie = 0, carry_sel = 0;
     for (int base = 0; base < nwords; base += G::NT) {
         const int wi = base + gtid;
@@ -722,6 +708,27 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
         carry_sel += tot;
     }
     G::sync();
+}
+
+// Stages a5 and a6 for one unit from a finished selection: ascending index list from the bitmap(s),
+// alpha, gather of the selected K and V rows with online softmax, combine with v_bar.
+// RG: gathered K and V rows in flight per half-warp (register budget of the calling kernel).
+// realloc = false leaves Step 3 out (out = the restricted attention; alpha is still reported).
+// Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
+// group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
+template <class G, int RG>
+__device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, SelectResult sel,
+                                       const PostScratch& sc, int k, const sparq_half* __restrict__ K_head,
+                                       const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
+                                       sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
+                                       float* __restrict__ alpha_out, bool build_list = true, bool realloc = true) {
+    const int n = hm.n, k_eff = hm.k_eff;
+    const float vmax = unkey32(kmax);
+    const float c1 = hm.inv_tau * LOG2E;
+    const float Z = sel.Z;
+    POST_CLK_INIT();
+    if (build_list) build_index_list<G>(gtid, hm, sel, sc);  // (a caller that kept sc.i2 from an earlier call skips the rebuild)
+    else G::sync();
     // start the selected rows on their way from HBM to L2 now; the gather below reads them a few
     // barriers later (two 128-byte lines per row and tensor)
     for (int i = gtid; i < 4 * k_eff; i += G::NT) {

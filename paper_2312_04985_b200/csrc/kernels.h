@@ -44,7 +44,7 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
 // sparq_decode_grouped.cu: group-shared selection (one CTA per KV head)
 int grouped_slices(int groups, int S_max, int n_sm);
 size_t grouped_scratch_bytes(int B, int Hq, int Hkv, int S_max, int slices);
-size_t grouped_dynamic_smem(int S_max);
+size_t grouped_dynamic_smem(int S_max, int g, int k);
 cudaError_t launch_sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                         const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                         int r, int k, int realloc, sparq_half* out, int32_t* idx_r, int32_t* idx_k,

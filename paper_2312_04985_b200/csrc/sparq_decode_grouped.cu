@@ -50,6 +50,8 @@ struct GroupShared {
     int32_t i2[SPARQ_K_MAX];
     unsigned long long gkey[D];           // g1: ranking keys
     uint16_t qh[SPARQ_G_MAX][D + 8];      // per head: selected components' fp16 bits in i1 order
+    alignas(16) uint16_t q16[SPARQ_G_MAX][D];   // per head: the whole query, fp16 bits (g5)
+    float pL[SPARQ_G_MAX];                // per head: sum of the exact attention's softmax weights (g5)
     float inv_tau[SPARQ_G_MAX];
     uint32_t kmax[SPARQ_G_MAX];           // per head: largest chain, as a key
     float zsum[SPARQ_G_MAX];              // per head: softmax denominator relative to it
@@ -120,6 +122,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
 #pragma unroll
         for (int h = 0; h < G; ++h) {
             qbits[h] = q[q_row0 + (size_t)h * D + tid];
+            sh.q16[h][tid] = qbits[h];
             aq[h] = fabsf(__half2float(__ushort_as_half(qbits[h])));
             sum += fixed_abs(qbits[h]);
         }
@@ -315,26 +318,137 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         sel_res = select_generic<CTA, true>(tid, hm, keys_sum, smax, 0.f, sc, r, S_max, Kt_head);
 
     GCLK(4);
-    // ------------------------------------------------------------------ g5: per head alpha, attention, Step 3
+    // ------------------------------------------------------------------ g5: alpha, exact attention, Step 3 -- all heads at once
+    // Every selected K and V row is gathered once and serves the g heads: q.K for all heads per row
+    // (scores to shared memory), per-head softmax weights, then the weighted V sums.
     const sparq_half* K_head = K + (size_t)bk * S_max * D;
     const sparq_half* V_head = V + (size_t)bk * S_max * D;
-#pragma unroll 1
-    for (int h = 0; h < G; ++h) {
-        __syncthreads();                                     // the previous head is done with hm and the scratch
-        if (tid < D) {
-            const uint16_t hb = q[q_row0 + (size_t)h * D + tid];
-            hm.q16[tid] = hb;
-            hm.qf[tid] = __half2float(__ushort_as_half(hb));
-        }
-        if (tid == 0) hm.inv_tau = sh.inv_tau[h];
-        __syncthreads();
-        SelectResult sr;
-        sr.Z = sh.zsum[h];
-        sr.need_tie = sel_res.need_tie;
-        finish<CTA, 4>(tid, hm, ws_unit + (size_t)h * S_max, sh.kmax[h], sr, sc, k, K_head, V_head, vbar_head,
-                       out0 + (size_t)h * D, (h == 0 && idx_k) ? idx_k + (size_t)bk * k : nullptr,
-                       alpha0 ? alpha0 + h : nullptr, /*build_list=*/h == 0, /*realloc=*/realloc != 0);
+    build_index_list<CTA>(tid, hm, sel_res, sc);             // sc.i2 ascending; the select stage's scratch is dead from here
+    for (int i = tid; i < 4 * k_eff; i += NT) {              // the rows on their way from HBM to L2 meanwhile
+        const int t = min(max(sc.i2[i >> 2], 0), n - 1);
+        const sparq_half* row = ((i & 2) ? V_head : K_head) + (size_t)t * D + (i & 1) * (D / 2);
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(row));
     }
+    float* zsc = reinterpret_cast<float*>(dyn_smem);                      // [G][k_eff] scores, then weights
+    float* slab = zsc + ((G * k_eff + 3) & ~3);                           // [warps][G][D] partial V sums
+    float alpha[G];                                          // per head: approximate-score mass of the selected set (Step 3)
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        float part = 0.f;
+        for (int j = tid; j < k_eff; j += NT)
+            part += ex2((unkey32(__ldcg(ws_unit + (size_t)h * S_max + sc.i2[j])) - vmax[h]) * c1[h]);
+        // (numerator and denominator are fp32 sums taken in different orders: keep the mass a probability)
+        alpha[h] = fminf(group_sum<CTA>(part, sh.red, tid) / sh.zsum[h], 1.0f);
+    }
+    const int hw = tid >> 4, l16 = tid & 15;
+    constexpr int RG = G >= 8 ? 2 : 4;                       // gathered rows in flight per half-warp
+    {
+        const float qscale = rsqrtf((float)D) * LOG2E;
+        const uint4* Kh = reinterpret_cast<const uint4*>(K_head);
+        for (int jb = 0; jb < k_eff; jb += CTA::NHW * RG) {  // trip count uniform across the CTA
+            uint4 kv[RG];
+#pragma unroll
+            for (int u = 0; u < RG; ++u) {
+                const int t = min(max(sc.i2[min(jb + u * CTA::NHW + hw, k_eff - 1)], 0), n - 1);
+                kv[u] = ld_stream(Kh + (size_t)t * (D / 8) + l16);
+            }
+#pragma unroll
+            for (int u = 0; u < RG; ++u) {
+                const int j = jb + u * CTA::NHW + hw;
+                const uint32_t kw[4] = {kv[u].x, kv[u].y, kv[u].z, kv[u].w};
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                    const uint4 q8 = *reinterpret_cast<const uint4*>(&sh.q16[h][l16 * 8]);
+                    const uint32_t qw[4] = {q8.x, q8.y, q8.z, q8.w};
+                    float zz = 0.f, zz2 = 0.f;               // exact fp16 products, two fp32 chains
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        fma_h(zz, (uint16_t)(kw[e] & 0xffffu), (uint16_t)(qw[e] & 0xffffu));
+                        fma_h(zz2, (uint16_t)(kw[e] >> 16), (uint16_t)(qw[e] >> 16));
+                    }
+                    zz = (zz + zz2) * qscale;
+#pragma unroll
+                    for (int o = 8; o > 0; o >>= 1) zz += __shfl_xor_sync(FULL, zz, o);
+                    if (l16 == 0 && j < k_eff) zsc[h * k_eff + j] = zz;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int h = warp; h < G; h += CTA::NW) {                // per head: maximum, weights in place, their sum
+        float mx = -CUDART_INF_F;
+        for (int j = lane; j < k_eff; j += 32) mx = fmaxf(mx, zsc[h * k_eff + j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+        float l_ = 0.f;
+        for (int j = lane; j < k_eff; j += 32) { const float w_ = ex2(zsc[h * k_eff + j] - mx); zsc[h * k_eff + j] = w_; l_ += w_; }
+        l_ = warp_sum(l_);
+        if (lane == 0) sh.pL[h] = l_;
+    }
+    __syncthreads();
+    {
+        float acc[G][8];
+#pragma unroll
+        for (int h = 0; h < G; ++h)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[h][e] = 0.f;
+        const uint4* Vh = reinterpret_cast<const uint4*>(V_head);
+        for (int jb = 0; jb < k_eff; jb += CTA::NHW * RG) {
+            uint4 vv[RG];
+#pragma unroll
+            for (int u = 0; u < RG; ++u) {
+                const int t = min(max(sc.i2[min(jb + u * CTA::NHW + hw, k_eff - 1)], 0), n - 1);
+                vv[u] = ld_stream(Vh + (size_t)t * (D / 8) + l16);
+            }
+#pragma unroll
+            for (int u = 0; u < RG; ++u) {
+                const int j = jb + u * CTA::NHW + hw;
+                if (j < k_eff) {
+                    const __half2* vh = reinterpret_cast<const __half2*>(&vv[u]);
+                    float2 f[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) f[e] = __half22float2(vh[e]);
+#pragma unroll
+                    for (int h = 0; h < G; ++h) {
+                        const float w_ = zsc[h * k_eff + j];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            acc[h][2 * e] = fmaf(w_, f[e].x, acc[h][2 * e]);
+                            acc[h][2 * e + 1] = fmaf(w_, f[e].y, acc[h][2 * e + 1]);
+                        }
+                    }
+                }
+            }
+        }
+        // the two half-warps of a warp, then the warps through shared memory (fixed order: reproducible)
+#pragma unroll
+        for (int h = 0; h < G; ++h)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[h][e] += __shfl_xor_sync(FULL, acc[h][e], 16);
+        if (lane < 16) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float4* dst = reinterpret_cast<float4*>(slab + ((size_t)warp * G + h) * D + l16 * 8);
+                dst[0] = make_float4(acc[h][0], acc[h][1], acc[h][2], acc[h][3]);
+                dst[1] = make_float4(acc[h][4], acc[h][5], acc[h][6], acc[h][7]);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < G * D; i += NT) {                  // Eq. (10) per head (or Eq. (8) alone)
+        const int h = i / D, c = i % D;
+        float s_ = 0.f;
+#pragma unroll
+        for (int w = 0; w < CTA::NW; ++w) s_ += slab[((size_t)w * G + h) * D + c];
+        const float y3 = s_ / sh.pL[h];
+        float a_ = alpha[0];
+#pragma unroll
+        for (int hh = 1; hh < G; ++hh) a_ = (h == hh) ? alpha[hh] : a_;
+        const float vb = __half2float(__ushort_as_half(vbar_head[c]));
+        out0[i] = __half_as_ushort(__float2half_rn(realloc ? a_ * y3 + (1.f - a_) * vb : y3));
+        if (c == 0 && alpha0) alpha0[h] = a_;
+    }
+    if (idx_k) for (int j = tid; j < k; j += NT) idx_k[(size_t)bk * k + j] = (j < k_eff) ? sc.i2[j] : -1;
     GCLK(5);
 }
 
@@ -348,7 +462,7 @@ cudaError_t launch_g(const sparq_half* q, const sparq_half* K, const sparq_half*
     const int groups = B * Hkv;
     uint32_t* ws_part = ws + (size_t)groups * (G + 1) * S_max;
     unsigned int* ws_count = ws_part + (size_t)groups * slices * 2 * G;
-    const size_t dyn = grouped_dynamic_smem(S_max);
+    const size_t dyn = grouped_dynamic_smem(S_max, G, k);
     cudaError_t e = cudaFuncSetAttribute(sparq_grouped_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     if (slices > 1) {
@@ -372,7 +486,13 @@ extern "C" int sparq_debug_group_clocks(unsigned long long* out16, int reset) {
 }
 #endif
 
-size_t grouped_dynamic_smem(int S_max) { return (post_scratch_bytes(CTA::NHW, grouped_bm_words(S_max)) + 127) & ~(size_t)127; }
+// The select stages' scratch, or -- later, in the same space -- the fused last stage's scores [g][k]
+// and partial V sums [warps][g][d_h], whichever is larger.
+size_t grouped_dynamic_smem(int S_max, int g, int k) {
+    const size_t select_bytes = post_scratch_bytes(CTA::NHW, grouped_bm_words(S_max));
+    const size_t fused_bytes = ((((size_t)g * k + 3) & ~(size_t)3) + (size_t)CTA::NW * g * D) * sizeof(float);
+    return ((select_bytes > fused_bytes ? select_bytes : fused_bytes) + 127) & ~(size_t)127;
+}
 
 // Slices per group.  With at least one group per SM the groups are left whole: the stages after the
 // stream (one CTA per group) weigh too much for slicing to pay (measured on 256 groups: 84 us whole,
