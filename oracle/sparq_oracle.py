@@ -474,6 +474,54 @@ def sparq_decode_opt(q, K, V, seq_lens, r, k, tau_mode="l1", realloc=True, windo
     return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k)
 
 
+# The same settings for the grouped selection (Section 4, "Grouped query attention").  Here the
+# temperature does change the selection: the summed scores sum_h s_hat[h, t] weigh the heads'
+# logits through their softmax, which depends on tau.  The window reserves the l most recent
+# positions as above; the other places go to the largest summed scores among the older positions.
+def group_scores_opt(Q: np.ndarray, K: np.ndarray, i1: np.ndarray, n: int, tau_mode: str = "l1"):
+    """:func:`group_scores` with the temperature of :func:`temperature_variant` per head."""
+    Q = np.asarray(Q, dtype=F64)
+    g = Q.shape[0]
+    log_s = np.zeros((g, n), dtype=F64)
+    tau = np.zeros(g, dtype=F64)
+    Ksel = np.asarray(K[:n][:, i1], dtype=F64)
+    for h in range(g):
+        tau[h] = temperature_variant(Q[h], i1, tau_mode)
+        log_s[h] = log_softmax((Ksel @ Q[h][i1]) / tau[h])
+    return log_s, tau
+
+
+def group_top_k_window(log_s: np.ndarray, k: int, window: int):
+    """:func:`group_top_k` with the local window of :func:`top_k_window`: the l = min(window, k_eff)
+    most recent positions, and the k_eff - l older positions with the largest summed scores."""
+    log_s = np.asarray(log_s, dtype=F64)
+    g, n = log_s.shape
+    if window < 0:
+        raise ValueError("window must be >= 0")
+    k_eff = max(0, min(int(k), n))
+    if k_eff == 0:
+        return np.zeros(0, dtype=np.int64), np.zeros(g, dtype=F64), math.inf
+    l = min(int(window), k_eff)
+    n_old, k_old = n - l, k_eff - l
+    log_total = np.logaddexp.reduce(log_s, axis=0)
+    order = _desc_order(log_total[:n_old])
+    sel = np.sort(np.concatenate([order[:k_old], np.arange(n_old, n)])).astype(np.int64)
+    alpha = np.sum(np.exp(log_s[:, sel]), axis=1)
+    gap = math.inf if (k_old == 0 or k_old == n_old) else abs(float(log_total[order[k_old - 1]] - log_total[order[k_old]]))
+    return sel, alpha, gap
+
+
+def sparq_group_opt(Q, K, V, v_bar, n, r, k, tau_mode="l1", realloc=True, window=0):
+    """The grouped step for one KV head with the settings above; the defaults are :func:`sparq_group`."""
+    if n < 1:
+        raise ValueError("sequence length must be >= 1")
+    i1, gap_r = group_top_r(Q, r)
+    log_s, tau = group_scores_opt(Q, K, i1, n, tau_mode)
+    i2, alpha, gap_k = group_top_k_window(log_s, k, window)
+    out = group_from_i2(Q, K, V, v_bar, i2, alpha, realloc)
+    return dict(out=out, i1=i1, i2=i2, alpha=alpha, gap_r=gap_r, gap_k=gap_k, tau=tau, log_s=log_s)
+
+
 # --------------------------------------------------------------------------- cache
 def cache_append(K, Kt, V, seq_lens, k_new, v_new):
     """One generation step's cache update (Section 3, text around Eq. (3); Appendix "Storing K

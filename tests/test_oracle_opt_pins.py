@@ -176,3 +176,67 @@ def test_batched_opt_decode_matches_per_head_calls():
     ref = O.sparq_decode(q, K, V, seq, 4, 6)
     np.testing.assert_allclose(plain["out"], ref["out"], rtol=1e-12)
     assert plain["i2"].tolist() == ref["i2"].tolist()
+
+
+# --------------------------------------------------------------------------- grouped selection with the settings
+def rand_group(g, n, d=16):
+    Q = RNG.standard_normal((g, d))
+    Q[:, RNG.choice(d, 3, replace=False)] *= 4.0
+    return Q, RNG.standard_normal((n, d)), RNG.standard_normal((n, d))
+
+
+def test_group_defaults_are_the_plain_grouped_step_and_a_group_of_one_is_the_head():
+    for _ in range(10):
+        g, n, r, k = int(RNG.integers(1, 4)), int(RNG.integers(3, 50)), int(RNG.integers(1, 9)), int(RNG.integers(0, 10))
+        Q, K, V = rand_group(g, n)
+        vb = O.mean_value(V, n)
+        a, b = O.sparq_group_opt(Q, K, V, vb, n, r, k), O.sparq_group(Q, K, V, vb, n, r, k)
+        assert a["i1"].tolist() == b["i1"].tolist() and a["i2"].tolist() == b["i2"].tolist()
+        np.testing.assert_allclose(a["out"], b["out"], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(a["alpha"], b["alpha"], rtol=1e-12, atol=1e-300)
+    for mode in O.TAU_MODES:
+        for w in (0, 2, 5):
+            Q, K, V = rand_group(1, 30)
+            vb = O.mean_value(V, 30)
+            grp = O.sparq_group_opt(Q, K, V, vb, 30, 4, 5, mode, False, w)
+            one = O.sparq_head_opt(Q[0], K, V, vb, 30, 4, 5, mode, False, w)
+            assert grp["i2"].tolist() == one["i2"].tolist()
+            np.testing.assert_allclose(grp["out"][0], one["out"], rtol=1e-12)
+            assert grp["alpha"][0] == pytest.approx(one["alpha"], rel=1e-12)
+
+
+def test_group_window_brute_force_and_temperature_dependence():
+    """Among the size-k sets that contain the window the selected one carries the largest summed mass;
+    and unlike the single-head case the temperature can change the group's choice."""
+    changed = 0
+    for _ in range(25):
+        g, n = int(RNG.integers(2, 4)), int(RNG.integers(5, 10))
+        k = int(RNG.integers(1, n))
+        w = int(RNG.integers(0, k + 1))
+        r = int(RNG.integers(1, 5))
+        Q, K, V = rand_group(g, n, d=8)
+        sets = {}
+        for mode in O.TAU_MODES:
+            res = O.sparq_group_opt(Q, K, V, O.mean_value(V, n), n, r, k, mode, True, w)
+            s_hat = np.exp(res["log_s"])
+            recent = set(range(n - w, n))
+            best = max((S for S in itertools.combinations(range(n), k) if recent <= set(S)),
+                       key=lambda S: s_hat[:, list(S)].sum())
+            assert sorted(best) == res["i2"].tolist()
+            for h in range(g):
+                assert res["alpha"][h] == pytest.approx(s_hat[h, list(best)].sum(), rel=1e-12)
+                assert res["tau"][h] == pytest.approx(O.temperature_variant(Q[h], res["i1"], mode), rel=1e-15)
+            sets[mode] = res["i2"].tolist()
+        changed += len({tuple(v) for v in sets.values()}) > 1
+    assert changed > 0
+
+
+def test_group_full_window_is_sliding_window_attention_per_head():
+    g, n, d, k = 3, 40, 16, 6
+    Q, K, V = rand_group(g, n, d)
+    res = O.sparq_group_opt(Q, K, V, np.full(d, 1e6), n, 4, k, "sqrt_r", False, k)
+    assert res["i2"].tolist() == list(range(n - k, n))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.tensor(Q)[None, :, None, :], torch.tensor(K[n - k:])[None, None].expand(1, g, k, d),
+        torch.tensor(V[n - k:])[None, None].expand(1, g, k, d))[0, :, 0].numpy()
+    np.testing.assert_allclose(res["out"], ref, rtol=1e-10, atol=1e-12)
