@@ -234,6 +234,21 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
 size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
 
 /*
+ * sparq_decode_grouped_opt -- sparq_decode_grouped with the settings of sparq_decode_opt:
+ * tau_mode picks every head's temperature (here it can change i2 as well: the summed scores
+ * weigh the heads' logits through their softmax), realloc = 0 leaves Step 3 out, and the
+ * l_eff = min(window, k_eff) most recent positions always belong to the group's i2, the other
+ * places going to the largest summed scores among the older positions.  sparq_decode_grouped is
+ * this call with SPARQ_TAU_L1 and window = 0.  SPARQ_ERR_BAD_OPTION as for sparq_decode_opt.
+ */
+int sparq_decode_grouped_opt(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                             const sparq_half* vbar, const int32_t* seq_lens,
+                             int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                             int tau_mode, int realloc, int window,
+                             sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
  * sparq_decode_1xk -- sparq_decode for a cache that stores K once (no transposed copy Kt): the
  * variant the paper measures beside the K-stored-twice one (Section 6.1) and leaves open because
  * of the 50 % extra memory Kt costs.  Stage a2 reads whole rows of K (the r selected components

@@ -207,11 +207,11 @@ size_t sparq_grouped_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {
     return grouped_scratch_bytes(B, Hq, Hkv, S_max, grouped_slices(B * Hkv, S_max, device_sm_count()));
 }
 
-int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
-                         const sparq_half* vbar, const int32_t* seq_lens,
-                         int B, int Hq, int Hkv, int d, int S_max, int r, int k, int realloc,
-                         sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+static int grouped_with(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                        const sparq_half* vbar, const int32_t* seq_lens,
+                        int B, int Hq, int Hkv, int d, int S_max, int r, int k, uint32_t opts,
+                        sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                        void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
     if (!q || !K || !Kt || !V || !vbar || !seq_lens || !out) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     const int g = Hq / Hkv;
@@ -221,8 +221,29 @@ int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_h
     if (S_max > SPARQ_S_MAX_WORKSPACE || grouped_dynamic_smem(S_max, Hq / Hkv, k) + 16384 > (size_t)device_smem_optin()) return SPARQ_ERR_TOO_LONG;
     const int slices = grouped_slices(B * Hkv, S_max, device_sm_count());
     if (!workspace || workspace_bytes < grouped_scratch_bytes(B, Hq, Hkv, S_max, slices)) return SPARQ_ERR_WORKSPACE;
-    return rc(launch_sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, realloc, out, idx_r, idx_k,
+    return rc(launch_sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
                                           alpha, status, workspace, slices, (cudaStream_t)stream));
+}
+
+int sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                         const sparq_half* vbar, const int32_t* seq_lens,
+                         int B, int Hq, int Hkv, int d, int S_max, int r, int k, int realloc,
+                         sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    return grouped_with(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, pack_opts(SPARQ_TAU_L1, realloc != 0, 0), out,
+                        idx_r, idx_k, alpha, workspace, workspace_bytes, status, stream);
+}
+
+int sparq_decode_grouped_opt(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
+                             const sparq_half* vbar, const int32_t* seq_lens,
+                             int B, int Hq, int Hkv, int d, int S_max, int r, int k,
+                             int tau_mode, int realloc, int window,
+                             sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
+                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (tau_mode < SPARQ_TAU_L1 || tau_mode > SPARQ_TAU_SQRT_R || window < 0 || window > SPARQ_K_MAX)
+        return SPARQ_ERR_BAD_OPTION;
+    return grouped_with(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, pack_opts(tau_mode, realloc != 0, window), out,
+                        idx_r, idx_k, alpha, workspace, workspace_bytes, status, stream);
 }
 
 size_t dense_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max) {

@@ -47,7 +47,7 @@ size_t grouped_scratch_bytes(int B, int Hq, int Hkv, int S_max, int slices);
 size_t grouped_dynamic_smem(int S_max, int g, int k);
 cudaError_t launch_sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                         const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                        int r, int k, int realloc, sparq_half* out, int32_t* idx_r, int32_t* idx_k,
+                                        int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k,
                                         float* alpha, int32_t* status, void* scratch, int slices, cudaStream_t stream);
 
 // dense_decode.cu

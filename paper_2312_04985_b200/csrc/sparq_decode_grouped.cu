@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(NT, G >= 8 ? 1 : 2)
 sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                      const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
                      const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
-                     int Hkv, int S_max, int r, int k, int realloc, int bm_words, int slices,
+                     int Hkv, int S_max, int r, int k, uint32_t opts, int bm_words, int slices,
                      sparq_half* __restrict__ out, int32_t* __restrict__ idx_r, int32_t* __restrict__ idx_k,
                      float* __restrict__ alpha_out, int32_t* status, uint32_t* ws, uint32_t* ws_part,
                      unsigned int* ws_count) {
@@ -156,9 +156,9 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
         float l1_all = aq[h], l1_sel = sel ? aq[h] : 0.f;
         group_sum2<CTA>(l1_all, l1_sel, sh.red, tid);
         // (a head with no weight on the group's components has all-zero approximate logits: tau := 1)
-        if (tid == 0) sh.inv_tau[h] = (l1_all > 0.f && l1_sel > 0.f) ? rsqrtf((float)D * l1_sel / l1_all) : 1.0f;
+        if (tid == 0) sh.inv_tau[h] = opt_inv_tau(opts, l1_all, l1_sel, r);
     }
-    if (tid == 0) { hm.bh = bk; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; hm.l1_sel = 0.f; hm.n_sel = n; hm.k_sel = k_eff; }
+    if (tid == 0) { hm.bh = bk; hm.n = n; hm.k_eff = k_eff; hm.valid = 1; hm.l1_sel = 0.f; hm.inv_tau = 1.f; opt_set_window(hm, n, k_eff, opts); }
     __syncthreads();
     if (p == 0 && idx_r) for (int j = tid; j < r; j += NT) idx_r[(size_t)bk * r + j] = hm.i1[j];
 
@@ -314,8 +314,15 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     sc.i2 = sh.i2; sc.red = sh.red; sc.redu = sh.redu; sc.res = sh.res; sc.band = sh.band;
     SelectResult sel_res;
     // kabs = 0: no rounding-error band, only exactly equal keys compete (lowest positions win)
-    if (!select_prefilled<CTA, GFB, true, true>(tid, hm, keys_sum, smax, 0.f, 1.f, sc, hist1, r, S_max, Kt_head, sel_res))
-        sel_res = select_generic<CTA, true>(tid, hm, keys_sum, smax, 0.f, sc, r, S_max, Kt_head);
+    const bool windowed = hm.n_sel != hm.n;                  // (uniform) a local window is reserved inside the budget
+    if (hm.k_sel == 0) {                                     // the window takes the whole budget: nothing to rank
+        sel_res = select_nothing<CTA>(tid, hm, keys_sum, smax, sc);
+    } else {
+        if (windowed) window_unhist<CTA, GFB>(tid, hm, keys_sum, hist1);
+        if (!select_prefilled<CTA, GFB, true, true>(tid, hm, keys_sum, smax, 0.f, 1.f, sc, hist1, r, S_max, Kt_head, sel_res))
+            sel_res = select_generic<CTA, true>(tid, hm, keys_sum, smax, 0.f, sc, r, S_max, Kt_head);
+    }
+    if (windowed) window_mark<CTA>(tid, hm, sc);
 
     GCLK(4);
     // ------------------------------------------------------------------ g5: alpha, exact attention, Step 3 -- all heads at once
@@ -445,7 +452,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
 #pragma unroll
         for (int hh = 1; hh < G; ++hh) a_ = (h == hh) ? alpha[hh] : a_;
         const float vb = __half2float(__ushort_as_half(vbar_head[c]));
-        out0[i] = __half_as_ushort(__float2half_rn(realloc ? a_ * y3 + (1.f - a_) * vb : y3));
+        out0[i] = __half_as_ushort(__float2half_rn(opt_realloc(opts) ? a_ * y3 + (1.f - a_) * vb : y3));
         if (c == 0 && alpha0) alpha0[h] = a_;
     }
     if (idx_k) for (int j = tid; j < k; j += NT) idx_k[(size_t)bk * k + j] = (j < k_eff) ? sc.i2[j] : -1;
@@ -456,7 +463,7 @@ int grouped_bm_words(int S_max) { return (S_max + 127) / 128 * 4; }
 
 template <int G>
 cudaError_t launch_g(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
-                     const sparq_half* vbar, const int32_t* seq_lens, int B, int Hkv, int S_max, int r, int k, int realloc,
+                     const sparq_half* vbar, const int32_t* seq_lens, int B, int Hkv, int S_max, int r, int k, uint32_t opts,
                      sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha, int32_t* status, uint32_t* ws,
                      int slices, cudaStream_t stream) {
     const int groups = B * Hkv;
@@ -469,7 +476,7 @@ cudaError_t launch_g(const sparq_half* q, const sparq_half* K, const sparq_half*
         e = cudaMemsetAsync(ws_count, 0, (size_t)groups * sizeof(unsigned int), stream);
         if (e != cudaSuccess) return e;
     }
-    sparq_grouped_kernel<G><<<(unsigned)slices * (unsigned)groups, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hkv, S_max, r, k, realloc,
+    sparq_grouped_kernel<G><<<(unsigned)slices * (unsigned)groups, NT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hkv, S_max, r, k, opts,
                                                                       grouped_bm_words(S_max), slices, out, idx_r, idx_k,
                                                                       alpha, status, ws, ws_part, ws_count);
     return cudaGetLastError();
@@ -514,14 +521,14 @@ size_t grouped_scratch_bytes(int B, int Hq, int Hkv, int S_max, int slices) {
 
 cudaError_t launch_sparq_decode_grouped(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                         const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
-                                        int r, int k, int realloc, sparq_half* out, int32_t* idx_r, int32_t* idx_k,
+                                        int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k,
                                         float* alpha, int32_t* status, void* scratch, int slices, cudaStream_t stream) {
     uint32_t* ws = static_cast<uint32_t*>(scratch);
     switch (Hq / Hkv) {
-        case 1: return launch_g<1>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, realloc, out, idx_r, idx_k, alpha, status, ws, slices, stream);
-        case 2: return launch_g<2>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, realloc, out, idx_r, idx_k, alpha, status, ws, slices, stream);
-        case 4: return launch_g<4>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, realloc, out, idx_r, idx_k, alpha, status, ws, slices, stream);
-        case 8: return launch_g<8>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, realloc, out, idx_r, idx_k, alpha, status, ws, slices, stream);
+        case 1: return launch_g<1>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha, status, ws, slices, stream);
+        case 2: return launch_g<2>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha, status, ws, slices, stream);
+        case 4: return launch_g<4>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha, status, ws, slices, stream);
+        case 8: return launch_g<8>(q, K, Kt, V, vbar, seq_lens, B, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha, status, ws, slices, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -30,7 +30,7 @@ HEAD_DIM = 128
 EXPORTS = ("sparq_status_string", "sparq_max_seq_len", "sparq_cache_build", "sparq_cache_append", "sparq_decode",
            "sparq_workspace_bytes", "dense_decode", "dense_workspace_bytes", "dense_decode_static", "sparq_step_host",
            "sparq_step_host_staging_bytes", "sparq_decode_grouped", "sparq_grouped_workspace_bytes",
-           "sparq_decode_1xk", "sparq_1xk_workspace_bytes", "sparq_decode_opt")
+           "sparq_decode_1xk", "sparq_1xk_workspace_bytes", "sparq_decode_opt", "sparq_decode_grouped_opt")
 
 
 class SparqError(RuntimeError):
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.sparq_step_host_staging_bytes.argtypes = [i] * 7
         L.sparq_decode_grouped.restype = i
         L.sparq_decode_grouped.argtypes = [vp] * 6 + [i] * 8 + [vp] * 4 + [vp, sz, vp, vp]
+        L.sparq_decode_grouped_opt.restype = i
+        L.sparq_decode_grouped_opt.argtypes = [vp] * 6 + [i] * 10 + [vp] * 4 + [vp, sz, vp, vp]
         L.sparq_grouped_workspace_bytes.restype = sz
         L.sparq_grouped_workspace_bytes.argtypes = [i] * 5
         L.sparq_decode_1xk.restype = i
@@ -203,6 +205,24 @@ def sparq_decode_grouped(q, K, Kt, V, vbar, seq_lens, r, k, out, workspace, real
                                         0 if workspace is None else workspace.numel() * workspace.element_size(),
                                         _dev(status, torch.int32, "status"), _stream(q))
     _check("sparq_decode_grouped", rc)
+    return out
+
+
+def sparq_decode_grouped_opt(q, K, Kt, V, vbar, seq_lens, r, k, out, workspace, tau_mode=TAU_L1, realloc=True, window=0,
+                             idx_r=None, idx_k=None, alpha=None, status=None):
+    B, Hq, d = q.shape
+    Hkv, S_max = K.shape[1], K.shape[2]
+    with torch.cuda.device(q.device):
+        rc = lib().sparq_decode_grouped_opt(_dev(q, torch.float16, "q"), _dev(K, torch.float16, "K"),
+                                            _dev(Kt, torch.float16, "Kt"), _dev(V, torch.float16, "V"),
+                                            _dev(vbar, torch.float16, "vbar"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                            B, Hq, Hkv, d, S_max, int(r), int(k), int(tau_mode), 1 if realloc else 0,
+                                            int(window), _dev(out, torch.float16, "out"), _dev(idx_r, torch.int32, "idx_r"),
+                                            _dev(idx_k, torch.int32, "idx_k"), _dev(alpha, torch.float32, "alpha"),
+                                            None if workspace is None else workspace.data_ptr(),
+                                            0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                            _dev(status, torch.int32, "status"), _stream(q))
+    _check("sparq_decode_grouped_opt", rc)
     return out
 
 

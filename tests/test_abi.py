@@ -66,6 +66,10 @@ def test_host_visible_errors_need_no_device(lib):
         assert opt(tau, 1, window) == sparq.ERR_BAD_OPTION
     assert opt(2, 0, 5, q=n) == sparq.ERR_NULL_POINTER
     assert opt(2, 0, 5, r=0) == sparq.ERR_BAD_RK
+    gopt = lambda tau, window: lib.sparq_decode_grouped_opt(
+        one, one, one, one, one, one, 1, 2, 1, 128, 8, 1, 1, tau, 1, window, one, n, n, n, one, 1 << 20, n, n)
+    for tau, window in ((3, 0), (0, -1), (0, sparq.K_MAX + 1)):
+        assert gopt(tau, window) == sparq.ERR_BAD_OPTION
     # a tensor pointer that is not 16-byte aligned (the kernels would fault on it)
     odd = ctypes.c_void_p(24)
     assert lib.sparq_decode(one, one, odd, one, one, one, 1, 1, 1, 128, 8, 1, 1, one, n, n, n, n, 0, n, n) == sparq.ERR_ALIGNMENT

@@ -35,7 +35,10 @@ def group_tolerance(Q, Kf, i1, tau, log_s, r):
     return GROUP_GAP_BASE + tol
 
 
-def run_grouped(cache, q, r, k, realloc=True):
+TAU = {sparq.TAU_L1: "l1", sparq.TAU_SQRT_D: "sqrt_d", sparq.TAU_SQRT_R: "sqrt_r"}
+
+
+def run_grouped(cache, q, r, k, realloc=True, tau_mode=None, window=0):
     q = q.to(cache.K.device).contiguous()
     B, Hq, d = q.shape
     Hkv = cache.Hkv
@@ -45,14 +48,19 @@ def run_grouped(cache, q, r, k, realloc=True):
     alpha = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=q.device)
     ws = torch.empty(max(16, sparq.sparq_grouped_workspace_bytes(B, Hq, Hkv, d, cache.S_max)), dtype=torch.uint8,
                      device=q.device)
-    sparq.sparq_decode_grouped(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, r, k, out, ws, realloc=realloc,
-                               idx_r=idx_r, idx_k=idx_k if k > 0 else None, alpha=alpha, status=cache.status)
+    if tau_mode is None and window == 0:
+        sparq.sparq_decode_grouped(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, r, k, out, ws, realloc=realloc,
+                                   idx_r=idx_r, idx_k=idx_k if k > 0 else None, alpha=alpha, status=cache.status)
+    else:
+        sparq.sparq_decode_grouped_opt(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, r, k, out, ws,
+                                       tau_mode=tau_mode or sparq.TAU_L1, realloc=realloc, window=window, idx_r=idx_r,
+                                       idx_k=idx_k if k > 0 else None, alpha=alpha, status=cache.status)
     torch.cuda.synchronize()
     return dict(out=out.cpu().numpy().astype(np.float64), i1=idx_r.cpu().numpy(), i2=idx_k.cpu().numpy(),
                 alpha=alpha.cpu().numpy().astype(np.float64))
 
 
-def compare_groups(gpu, q, K, V, seq, r, k, realloc=True, what=""):
+def compare_groups(gpu, q, K, V, seq, r, k, realloc=True, what="", tau_mode=None, window=0):
     """Every (batch, KV head) group against the oracle.  q [B,Hq,d], K/V [B,Hkv,S,d] fp16 numpy."""
     B, Hq, d = q.shape
     Hkv = K.shape[1]
@@ -65,8 +73,9 @@ def compare_groups(gpu, q, K, V, seq, r, k, realloc=True, what=""):
             Q = q[b, hkv * g:(hkv + 1) * g].astype(np.float64)
             Kf, Vf = K[b, hkv, :n].astype(np.float64), V[b, hkv, :n].astype(np.float64)
             vb = O.mean_value(Vf, n)
-            ora = O.sparq_group(Q, Kf, Vf, vb, n, r, k, realloc)
+            ora = O.sparq_group_opt(Q, Kf, Vf, vb, n, r, k, TAU[tau_mode or sparq.TAU_L1], realloc, window)
             k_eff = min(k, n)
+            l_eff = min(window, k_eff)
             np.testing.assert_array_equal(gpu["i1"][b, hkv], ora["i1"], err_msg=tag)
             got_i2 = gpu["i2"][b, hkv][:k_eff].astype(np.int64)
             assert (gpu["i2"][b, hkv][k_eff:] == -1).all(), tag + ": idx_k tail must be -1"
@@ -76,8 +85,9 @@ def compare_groups(gpu, q, K, V, seq, r, k, realloc=True, what=""):
                 assert 0 < ora["gap_k"] < tol, tag + ": i2 differs, gap_k=%g, tolerance %g" % (ora["gap_k"], tol)
                 assert len(set(got_i2.tolist())) == k_eff and got_i2.min() >= 0 and got_i2.max() < n, tag
                 assert (np.diff(got_i2) > 0).all(), tag + ": idx_k must ascend"
+                assert set(range(n - l_eff, n)) <= set(got_i2.tolist()), tag + ": the window must be selected"
                 log_total = np.logaddexp.reduce(ora["log_s"], axis=0)
-                thr = np.sort(log_total)[::-1][k_eff - 1]
+                thr = np.sort(log_total[:n - l_eff])[::-1][k_eff - l_eff - 1]
                 for t in set(got_i2.tolist()) ^ set(ora["i2"].tolist()):     # only positions at the threshold may swap
                     assert abs(log_total[t] - thr) <= tol, tag
                 want_alpha = np.exp(ora["log_s"][:, got_i2]).sum(axis=1)
@@ -183,3 +193,46 @@ def test_grouped_bad_length_and_host_errors():
         sparq.sparq_decode_grouped(q[:, :24].contiguous(), cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, 16, 8,
                                    out[:, :24].contiguous(), torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
     assert e.value.code == sparq.ERR_BAD_SHAPE
+
+
+SETTINGS = [
+    (sparq.TAU_SQRT_D, True, 0),
+    (sparq.TAU_SQRT_R, False, 0),
+    (sparq.TAU_L1, True, 32),          # the paper's l = k/4 at k = 128
+    (sparq.TAU_SQRT_R, True, 37),      # a window that starts and ends inside bitmap words
+    (sparq.TAU_L1, False, 128),        # the window takes the whole budget
+    (sparq.TAU_SQRT_D, True, 500),     # larger than k: clipped
+]
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("c3", dict(B=2, S=4096, ragged=(90, 4000))),                     # g = 4, whole groups; one sequence may be shorter than k
+    ("c3", dict(B=1, S=16384, Hq=8, Hkv=2)),                          # two groups over a long cache: sliced, tickets
+    ("c3", dict(B=1, S=2048, Hq=16, Hkv=2)),                          # g = 8
+])
+def test_grouped_settings_against_oracle(name, kw):
+    c = synth.make_case(name, backend="numpy", **kw)
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens + c.n_steps)
+    q, K, V, seq = _case_arrays(c)
+    for tau_mode, realloc, window in SETTINGS:
+        gpu = run_grouped(cache, c.q_steps[-1], c.r, c.k, realloc=realloc, tau_mode=tau_mode, window=window)
+        waived = compare_groups(gpu, q, K, V, seq, c.r, c.k, realloc=realloc, tau_mode=tau_mode, window=window,
+                                what="%s %s tau=%d realloc=%d window=%d" % (name, kw, tau_mode, realloc, window))
+        assert waived <= max(1, c.B * c.Hkv // 8)
+    cache.check_status(0)
+
+
+def test_grouped_opt_defaults_and_bad_options():
+    c = synth.make_case("c3", backend="numpy", B=2, S=1024)
+    cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
+    a = run_grouped(cache, c.q_steps[0], c.r, c.k)
+    b = run_grouped(cache, c.q_steps[0], c.r, c.k, tau_mode=sparq.TAU_L1, window=0)
+    for key in ("out", "i1", "i2", "alpha"):
+        np.testing.assert_array_equal(a[key], b[key])
+    q = c.q_steps[0].cuda()
+    ws = torch.empty(1 << 22, dtype=torch.uint8, device="cuda")
+    for kw in (dict(tau_mode=3), dict(window=-1), dict(window=sparq.K_MAX + 1)):
+        with pytest.raises(sparq.SparqError) as e:
+            sparq.sparq_decode_grouped_opt(q, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, 16, 8,
+                                           torch.empty_like(q), ws, **kw)
+        assert e.value.code == sparq.ERR_BAD_OPTION
