@@ -451,9 +451,9 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // keys builds the bitmap of everything above the threshold bin, the softmax denominator and the list
 // of the bin's own keys; the threshold is then resolved inside that short list, and the 2B band
 // around it re-decided in fp64 as in select_generic.  Clears hist1 for its next user (not with WIDE).
-// Returns false (for every thread of the group alike) when the short-cut does not apply -- a warp
-// meets more of the bin's keys than its list segment holds, or the band reaches outside the bin or holds too many keys -- and
-// the caller runs select_generic instead.
+// Returns false (for every thread of the group alike) when the short-cut does not apply -- the bin
+// holds more keys than the list (with WIDE) or a warp's segment of it (without) has room for, or the
+// band reaches outside the bin or holds too many keys -- and the caller runs select_generic instead.
 // Z_stream: the softmax denominator relative to the largest key, accumulated by the stream stage.
 template <class G, int FB_ = FB, bool WIDE = false, bool BY_POS = false>
 __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
@@ -483,43 +483,47 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const int nwords = (n + 31) >> 5;
     uint32_t wcount = 0;                                     // this warp's list length (warp-uniform)
     if constexpr (WIDE) {
-        // Keys in global memory: one 16-byte vector per lane and load, four loads in flight, so that a
-        // warp has 2 KB on its way instead of 512 bytes.  A warp covers 128 positions (four bitmap
-        // words) per load: lane l holds positions 4l .. 4l+3 of the group, i.e. nibble l % 8 of
-        // bitmap word l / 8, and the eight lanes of a word OR their nibbles together.
-        const int ngroups = (n + 127) >> 7;
-        const unsigned oct = 0xffu << (lane & 24);           // the eight lanes that share a bitmap word
-        for (int g0 = warp; g0 < ngroups; g0 += 4 * G::NW) {
-            uint4 kv[4];
+        // Keys in global memory.  A lane owns eight consecutive positions -- two 16-byte loads and one
+        // whole byte of the bitmap, so no lane talks to another -- and a warp 256 positions per step,
+        // two steps in flight.  The bin's own keys are rare: a lane that meets some reserves their
+        // places in the one list of the group with a single shared-memory atomic.  (With one warp
+        // per scheduler, as in the 128-thread kernels, this scan is bound by its own instruction
+        // stream, not by the loads: issuing every load twice changed its time by 5 %.)
+        unsigned char* bm8 = reinterpret_cast<unsigned char*>(sc.bm_sel);
+        uint32_t* list_key = sc.hist;
+        int32_t* list_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX);
+        const int nblocks = (n + 255) >> 8;
+        for (int b0 = warp; b0 < nblocks; b0 += 2 * G::NW) {
+            uint4 kv[2][2];
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int t = ((g0 + x * G::NW) << 7) + lane * 4;
-                kv[x] = t < n ? *reinterpret_cast<const uint4*>(keys + t) : make_uint4(0u, 0u, 0u, 0u);
+            for (int x = 0; x < 2; ++x) {
+                const int t = ((b0 + x * G::NW) << 8) + lane * 8;        // a multiple of 8: both vectors lie inside the buffer
+                kv[x][0] = t < n ? *reinterpret_cast<const uint4*>(keys + t) : make_uint4(0u, 0u, 0u, 0u);
+                kv[x][1] = t < n ? *reinterpret_cast<const uint4*>(keys + t + 4) : make_uint4(0u, 0u, 0u, 0u);
             }
 #pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int gi = g0 + x * G::NW;
-                if (gi < ngroups) {                          // warp-uniform
-                    const int t = (gi << 7) + lane * 4;
-                    const uint32_t u[4] = {kv[x].x, kv[x].y, kv[x].z, kv[x].w};
-                    uint32_t nib = 0, inb = 0;
+            for (int x = 0; x < 2; ++x) {
+                const int t = ((b0 + x * G::NW) << 8) + lane * 8;
+                if (t < nwords * 32) {                       // (the bytes of the last word past n are written too, as zeros)
+                    const uint32_t u[8] = {kv[x][0].x, kv[x][0].y, kv[x][0].z, kv[x][0].w, kv[x][1].x, kv[x][1].y, kv[x][1].z, kv[x][1].w};
+                    uint32_t sel8 = 0, inb = 0;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const bool valid = t + e < n;
+                    for (int e = 0; e < 8; ++e) {
                         const uint32_t dig = u[e] >> FSH_;
-                        nib |= (valid && dig > b1) ? 1u << e : 0u;
-                        inb |= (valid && dig == b1) ? 1u << e : 0u;
+                        sel8 |= (dig > b1) ? 1u << e : 0u;
+                        inb |= (dig == b1) ? 1u << e : 0u;
                     }
-                    const uint32_t word = __reduce_or_sync(oct, nib << ((lane & 7) * 4));
-                    const int wi = (gi << 2) + (lane >> 3);
-                    if ((lane & 7) == 0 && wi < nwords) sc.bm_sel[wi] = word;
-                    if (__any_sync(FULL, inb != 0)) {        // the bin's own keys go to the warp's list
+                    const int rem = n - t;                   // valid positions among the eight
+                    if (rem < 8) { const uint32_t vm = rem > 0 ? (1u << rem) - 1u : 0u; sel8 &= vm; inb &= vm; }
+                    bm8[t >> 3] = (unsigned char)sel8;
+                    if (inb) {
+                        uint32_t slot = atomicAdd(&sc.band[3], (uint32_t)__popc(inb));
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const unsigned be = __ballot_sync(FULL, inb >> e & 1u);
-                            const uint32_t slot = wcount + __popc(be & lt);
-                            if ((inb >> e & 1u) && slot < SEG) { seg_key[slot] = u[e]; seg_pos[slot] = t + e; }
-                            wcount += __popc(be);
+                        for (int e = 0; e < 8; ++e) {
+                            if ((inb >> e) & 1u) {
+                                if (slot < (uint32_t)LIST_MAX) { list_key[slot] = u[e]; list_pos[slot] = t + e; }
+                                ++slot;
+                            }
                         }
                     }
                 }
@@ -560,10 +564,19 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     POST_CLK(1);
     uint32_t m = 0;
     bool fits = true;
+    if constexpr (WIDE) {
+        m = sc.band[3];
+        fits = m <= (uint32_t)LIST_MAX;
+    } else {
 #pragma unroll
-    for (int w = 0; w < G::NW; ++w) { const uint32_t c = sc.redu[G::NW + w]; m += c; fits = fits && c <= SEG; }
+        for (int w = 0; w < G::NW; ++w) { const uint32_t c = sc.redu[G::NW + w]; m += c; fits = fits && c <= SEG; }
+    }
     if (!fits) return false;
-    const uint32_t my_n = min(wcount, (uint32_t)SEG);
+    // this thread's walk over the list(s): its warp's segment, or its share of the group's one list
+    const uint32_t* my_key = WIDE ? sc.hist : seg_key;
+    const int32_t* my_pos = WIDE ? reinterpret_cast<const int32_t*>(sc.hist + LIST_MAX) : seg_pos;
+    const uint32_t my_first = WIDE ? (uint32_t)gtid : (uint32_t)lane, my_step = WIDE ? (uint32_t)G::NT : 32u;
+    const uint32_t my_n = WIDE ? m : min(wcount, (uint32_t)SEG);
 
     // the threshold among the bin's m keys: `need` of them are wanted; remaining bits as 8 + 8 + the rest
     uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH_, mask = ~0u << FSH_, ceq = m;
@@ -581,8 +594,8 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         const int bits = pass < 2 ? 8 : FSH_ - 16;
         shift -= bits;
         uint32_t* hcur = h256 + pass * 256;
-        for (uint32_t i = lane; i < my_n; i += 32) {
-            const uint32_t u = seg_key[i];
+        for (uint32_t i = my_first; i < my_n; i += my_step) {
+            const uint32_t u = my_key[i];
             if ((u & mask) == prefix) atomicAdd(&hcur[(u >> shift) & ((1u << bits) - 1)], 1u);
         }
         G::sync();
@@ -619,9 +632,9 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
     if ((lo_key >> FSH_) != b1 || (hi_key >> FSH_) != b1) return false;   // keys outside the list may be in the band
 
-    for (uint32_t i = lane; i < my_n; i += 32) {
-        const uint32_t u = seg_key[i];
-        const int t = seg_pos[i];
+    for (uint32_t i = my_first; i < my_n; i += my_step) {
+        const uint32_t u = my_key[i];
+        const int t = my_pos[i];
         if (u >= edge) atomicOr(&sc.bm_sel[t >> 5], 1u << (t & 31));
         if (u >= lo_key && u <= hi_key) {
             atomicAdd(&sc.band[u >= edge ? 1 : 0], 1u);
@@ -738,7 +751,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     }
     // alpha = approximate-score mass of the selected set (Step 3)
     float apart = 0.f;
-    for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[sc.i2[j]]) - vmax) * c1);
+    for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[min(max(sc.i2[j], 0), n - 1)]) - vmax) * c1);
     // (numerator and denominator are fp32 sums taken in different orders: keep the mass a probability)
     const float alpha = fminf(group_sum<G>(apart, sc.red, gtid) / Z, 1.0f);
     POST_CLK(4);

@@ -343,7 +343,7 @@ sparq_grouped_kernel(const sparq_half* __restrict__ q, const sparq_half* __restr
     for (int h = 0; h < G; ++h) {
         float part = 0.f;
         for (int j = tid; j < k_eff; j += NT)
-            part += ex2((unkey32(__ldcg(ws_unit + (size_t)h * S_max + sc.i2[j])) - vmax[h]) * c1[h]);
+            part += ex2((unkey32(__ldcg(ws_unit + (size_t)h * S_max + min(max(sc.i2[j], 0), n - 1))) - vmax[h]) * c1[h]);
         // (numerator and denominator are fp32 sums taken in different orders: keep the mass a probability)
         alpha[h] = fminf(group_sum<CTA>(part, sh.red, tid) / sh.zsum[h], 1.0f);
     }
