@@ -445,6 +445,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
 
 // First-digit histogram the stream stage fills while the keys are still in registers.
 constexpr int FB = 10, FSH = 32 - FB, FBINS = 1 << FB;
+constexpr int WIDE_DEPTH = 4;            // 256-position steps in flight per warp in the scan of keys in global memory (2: 2 % slower on c3; 8: no better)
 constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the threshold bin; the list lives in sc.hist
 
 // Stages a4 + a3 when hist1 already holds the histogram of the keys' top FB bits.  One scan of the
@@ -485,7 +486,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     if constexpr (WIDE) {
         // Keys in global memory.  A lane owns eight consecutive positions -- two 16-byte loads and one
         // whole byte of the bitmap, so no lane talks to another -- and a warp 256 positions per step,
-        // two steps in flight.  The bin's own keys are rare: a lane that meets some reserves their
+        // WIDE_DEPTH steps in flight.  The bin's own keys are rare: a lane that meets some reserves their
         // places in the one list of the group with a single shared-memory atomic.  (With one warp
         // per scheduler, as in the 128-thread kernels, this scan is bound by its own instruction
         // stream, not by the loads: issuing every load twice changed its time by 5 %.)
@@ -493,16 +494,16 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
         uint32_t* list_key = sc.hist;
         int32_t* list_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX);
         const int nblocks = (n + 255) >> 8;
-        for (int b0 = warp; b0 < nblocks; b0 += 2 * G::NW) {
-            uint4 kv[2][2];
+        for (int b0 = warp; b0 < nblocks; b0 += WIDE_DEPTH * G::NW) {
+            uint4 kv[WIDE_DEPTH][2];
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
+            for (int x = 0; x < WIDE_DEPTH; ++x) {
                 const int t = ((b0 + x * G::NW) << 8) + lane * 8;        // a multiple of 8: both vectors lie inside the buffer
                 kv[x][0] = t < n ? *reinterpret_cast<const uint4*>(keys + t) : make_uint4(0u, 0u, 0u, 0u);
                 kv[x][1] = t < n ? *reinterpret_cast<const uint4*>(keys + t + 4) : make_uint4(0u, 0u, 0u, 0u);
             }
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
+            for (int x = 0; x < WIDE_DEPTH; ++x) {
                 const int t = ((b0 + x * G::NW) << 8) + lane * 8;
                 if (t < nwords * 32) {                       // (the bytes of the last word past n are written too, as zeros)
                     const uint32_t u[8] = {kv[x][0].x, kv[x][0].y, kv[x][0].z, kv[x][0].w, kv[x][1].x, kv[x][1].y, kv[x][1].z, kv[x][1].w};
