@@ -535,9 +535,13 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
 }
 
 // Slices per unit of the split plan: enough CTAs for about two waves of resident CTAs, at least
-// one pass of SCH positions per slice; 0 when the plan does not apply (a short cache).
+// one pass of SCH positions per slice; 0 when the plan does not apply (a short cache).  With two
+// or more whole units per SM the units are left whole: slicing then only adds the repeated top-r
+// and the merge of the slices (1024 units of 16384 positions: 146 us whole, 154 us in two slices,
+// 151 in three; 512 units of up to 32800: 287 whole, 290 in three).
 int split_count(int units, int S_max, int n_sm) {
     if (n_sm <= 0 || S_max < 2 * SCH) return 0;
+    if (units >= 2 * n_sm) return 1;
     const int want = (2 * SPLIT_CTAS * n_sm + units - 1) / units;      // about two waves of resident CTAs
     const int cap = (S_max + SCH - 1) / SCH;
     const int s = want < cap ? want : cap;
