@@ -266,7 +266,9 @@ size_t sparq_1xk_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max);
  * sparq_step_host -- one whole generation step driven from HOST buffers: copies q_host
  * [B,Hq,d], k_new_host and v_new_host [B,Hkv,d] (fp16, ideally pinned) to the device, runs
  * sparq_cache_append then sparq_decode on `stream`, copies the result to out_host [B,Hq,d]
- * and waits for the stream.  The cache (K, Kt, V, vsum, vbar, seq_lens) stays resident on the
+ * and waits for the stream.  With k_new_host and v_new_host both NULL, q_host is one buffer
+ * that holds q, k_new and v_new back to back (in that order), and they travel in one copy
+ * instead of three.  The cache (K, Kt, V, vsum, vbar, seq_lens) stays resident on the
  * device.  staging: device scratch of at least sparq_step_host_staging_bytes() bytes (device
  * copies of the four host tensors, then the workspace sparq_workspace_bytes() names for these
  * shapes, at least 64 bytes).

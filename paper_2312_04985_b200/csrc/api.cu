@@ -289,23 +289,28 @@ int sparq_step_host(const sparq_half* q_host, const sparq_half* k_new_host, cons
                     sparq_half* K, sparq_half* Kt, sparq_half* V, float* vsum, sparq_half* vbar,
                     int32_t* seq_lens, int B, int Hq, int Hkv, int d, int S_max, int r, int k,
                     sparq_half* out_host, void* staging, size_t staging_bytes, int32_t* status, void* stream) {
-    if (!q_host || !k_new_host || !v_new_host || !out_host) return SPARQ_ERR_NULL_POINTER;
+    const bool packed = !k_new_host && !v_new_host;          // q_host holds q, k_new, v_new back to back
+    if (!q_host || !out_host || (!packed && (!k_new_host || !v_new_host))) return SPARQ_ERR_NULL_POINTER;
     if (bad_common(B, Hq, Hkv, d, S_max)) return SPARQ_ERR_BAD_SHAPE;
     if (!staging || staging_bytes < sparq_step_host_staging_bytes(B, Hq, Hkv, d, S_max, r, k)) return SPARQ_ERR_WORKSPACE;
     if (misaligned(staging)) return SPARQ_ERR_ALIGNMENT;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t nq = (size_t)B * Hq * d, nkv = (size_t)B * Hkv * d;
-    sparq_half* q_dev = (sparq_half*)staging;
-    sparq_half* out_dev = q_dev + nq;
-    sparq_half* k_dev = out_dev + nq;
+    sparq_half* q_dev = (sparq_half*)staging;                // device copies: q | k_new | v_new | out
+    sparq_half* k_dev = q_dev + nq;
     sparq_half* v_dev = k_dev + nkv;
-    if (cudaMemcpyAsync(q_dev, q_host, nq * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(k_dev, k_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(v_dev, v_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    sparq_half* out_dev = v_dev + nkv;
+    if (packed) {                                            // one copy instead of three
+        if (cudaMemcpyAsync(q_dev, q_host, (nq + 2 * nkv) * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SPARQ_ERR_CUDA;
+    } else if (cudaMemcpyAsync(q_dev, q_host, nq * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+               cudaMemcpyAsync(k_dev, k_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+               cudaMemcpyAsync(v_dev, v_new_host, nkv * sizeof(sparq_half), cudaMemcpyHostToDevice, st) != cudaSuccess) {
         return SPARQ_ERR_CUDA;
+    }
     int code = sparq_cache_append(k_dev, v_dev, K, Kt, V, vsum, vbar, seq_lens, B, Hkv, d, S_max, status, stream);
     if (code != SPARQ_OK) return code;
-    void* ws = v_dev + nkv;                                  // the tail of the staging area: the decode's workspace
+    void* ws = out_dev + nq;                                 // the tail of the staging area: the decode's workspace
     code = sparq_decode(q_dev, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, d, S_max, r, k, out_dev, nullptr, nullptr, nullptr,
                         ws, step_host_ws_bytes(B, Hq, Hkv, d, S_max, r, k), status, stream);
     if (code != SPARQ_OK) return code;

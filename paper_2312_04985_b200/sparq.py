@@ -277,15 +277,24 @@ def dense_decode_static(q, K, V, seq_lens, out, status=None):
 
 def sparq_step_host(q_host, k_new_host, v_new_host, K, Kt, V, vsum, vbar, seq_lens, r, k, out_host, staging,
                     status=None):
-    """Host-buffer step: q_host, k_new_host, v_new_host, out_host are CPU (pinned) fp16 tensors."""
-    B, Hq, d = q_host.shape
-    Hkv, S_max = K.shape[1], K.shape[2]
+    """Host-buffer step: q_host, k_new_host, v_new_host, out_host are CPU (pinned) fp16 tensors.
+    With k_new_host = v_new_host = None, q_host is a flat buffer holding q [B,Hq,d], k_new and
+    v_new [B,Hkv,d] back to back (one copy to the device instead of three)."""
+    Hkv, S_max, d = K.shape[1], K.shape[2], K.shape[3]
+    B = out_host.shape[0]
+    Hq = out_host.shape[1]
+    packed = k_new_host is None and v_new_host is None
+    if packed and q_host.numel() != B * (Hq + 2 * Hkv) * d:
+        raise ValueError("packed q_host must hold B*(Hq + 2*Hkv)*d elements")
     for t, name in ((q_host, "q_host"), (k_new_host, "k_new_host"), (v_new_host, "v_new_host"),
                     (out_host, "out_host")):
-        if t.is_cuda or t.dtype != torch.float16 or not t.is_contiguous():
+        if t is None and packed:
+            continue
+        if t is None or t.is_cuda or t.dtype != torch.float16 or not t.is_contiguous():
             raise ValueError("%s must be a contiguous CPU float16 tensor" % name)
     with torch.cuda.device(K.device):
-        rc = lib().sparq_step_host(q_host.data_ptr(), k_new_host.data_ptr(), v_new_host.data_ptr(),
+        rc = lib().sparq_step_host(q_host.data_ptr(), None if packed else k_new_host.data_ptr(),
+                                   None if packed else v_new_host.data_ptr(),
                                    _dev(K, torch.float16, "K"), _dev(Kt, torch.float16, "Kt"),
                                    _dev(V, torch.float16, "V"), _dev(vsum, torch.float32, "vsum"),
                                    _dev(vbar, torch.float16, "vbar"), _dev(seq_lens, torch.int32, "seq_lens"),

@@ -52,6 +52,13 @@ def test_host_visible_errors_need_no_device(lib):
     assert lib.dense_decode_static(one, one, one, one, 1, 1, 1, 128, 8, n, n, n) == sparq.ERR_NULL_POINTER
     assert lib.sparq_cache_append(one, one, one, one, one, one, one, n, 1, 1, 128, 8, n, n) == sparq.ERR_NULL_POINTER
     assert lib.sparq_cache_build(one, one, one, one, n, one, 1, 1, 128, 8, n, n) == sparq.ERR_NULL_POINTER
+    # the host-buffer step: k_new and v_new may be NULL only together (then q_host is the packed buffer)
+    step = lambda q, kn, vn, out: lib.sparq_step_host(q, kn, vn, one, one, one, one, one, one, 1, 1, 1, 128, 8, 1, 1, out, n, 0, n, n)
+    assert step(one, n, one, one) == sparq.ERR_NULL_POINTER
+    assert step(one, one, n, one) == sparq.ERR_NULL_POINTER
+    assert step(n, n, n, one) == sparq.ERR_NULL_POINTER
+    assert step(one, n, n, n) == sparq.ERR_NULL_POINTER
+    assert step(one, n, n, one) == sparq.ERR_WORKSPACE          # packed form accepted; refused next for its missing staging area
     # shapes: d != 128, Hq not a multiple of Hkv, S_max not a multiple of 8, B < 1
     for B, Hq, Hkv, d, S in ((1, 1, 1, 64, 8), (1, 3, 2, 128, 8), (1, 1, 1, 128, 12), (0, 1, 1, 128, 8)):
         assert lib.sparq_decode(one, one, one, one, one, one, B, Hq, Hkv, d, S, 1, 1, one, n, n, n, n, 0, n, n) == sparq.ERR_BAD_SHAPE

@@ -332,3 +332,21 @@ def test_step_host_matches_device_step():
                               b.K, b.Kt, b.V, b.vsum, b.vbar, b.seq_lens, c.r, c.k, out_host, staging, b.status)
         np.testing.assert_array_equal(out_host.numpy().astype(np.float64), ref["out"])
     assert torch.equal(a.Kt, b.Kt) and torch.equal(a.seq_lens, b.seq_lens)
+
+
+def test_step_host_with_inputs_back_to_back_in_one_buffer():
+    """q, k_new, v_new packed in one pinned buffer (k_new_host = v_new_host = NULL) travel in a single copy: same results."""
+    c = synth.make_case("c4", B=2, n_steps=2, ragged=(500, 900), Hq=8, Hkv=2, backend="numpy")
+    a = H.DeviceCache(c.K, c.V, c.seq_lens)
+    b = H.DeviceCache(c.K, c.V, c.seq_lens)
+    staging = torch.empty(sparq.sparq_step_host_staging_bytes(c.B, c.Hq, c.Hkv, c.d, c.S_max, c.r, c.k), dtype=torch.uint8, device="cuda")
+    out_host = torch.empty(c.B, c.Hq, c.d, dtype=torch.float16).pin_memory()
+    nq, nkv = c.B * c.Hq * c.d, c.B * c.Hkv * c.d
+    buf = torch.empty(nq + 2 * nkv, dtype=torch.float16).pin_memory()
+    for i in range(c.n_steps):
+        a.append(c.k_steps[i], c.v_steps[i])
+        ref = a.decode(c.q_steps[i], c.r, c.k)
+        buf[:nq].copy_(c.q_steps[i].reshape(-1)); buf[nq:nq + nkv].copy_(c.k_steps[i].reshape(-1)); buf[nq + nkv:].copy_(c.v_steps[i].reshape(-1))
+        sparq.sparq_step_host(buf, None, None, b.K, b.Kt, b.V, b.vsum, b.vbar, b.seq_lens, c.r, c.k, out_host, staging, b.status)
+        np.testing.assert_array_equal(out_host.numpy().astype(np.float64), ref["out"])
+    assert torch.equal(a.Kt, b.Kt) and torch.equal(a.V, b.V) and torch.equal(a.seq_lens, b.seq_lens)
