@@ -178,7 +178,7 @@ int sparq_decode_opt(const sparq_half* q, const sparq_half* K, const sparq_half*
 }
 
 static int one_k_splits(int units, int S_max) {
-    const int s = split_count(units, S_max, device_sm_count());
+    const int s = split_count(units, S_max, device_sm_count(), /*one_k=*/true);
     return s < 1 ? 1 : s;
 }
 

@@ -26,7 +26,7 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
 
 // split-S plan (sparq_decode.cu): one CTA per (slice, unit) with the keys in a scratch buffer, for
 // caches too long for the persistent kernel and for few units with long sequences
-int split_count(int units, int S_max, int n_sm);
+int split_count(int units, int S_max, int n_sm, bool one_k = false);
 size_t split_scratch_bytes(int units, int S_max, int splits);
 cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                       const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,

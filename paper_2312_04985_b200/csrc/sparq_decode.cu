@@ -539,9 +539,11 @@ cudaError_t launch_sparq_decode(const sparq_half* q, const sparq_half* K, const 
 // or more whole units per SM the units are left whole: slicing then only adds the repeated top-r
 // and the merge of the slices (1024 units of 16384 positions: 146 us whole, 154 us in two slices,
 // 151 in three; 512 units of up to 32800: 287 whole, 290 in three).
-int split_count(int units, int S_max, int n_sm) {
+// (The variant that stores K once reads d_h / r times the bytes per unit and keeps the slices:
+// 1024 such units took 1121 us whole against 885 us in two slices.)
+int split_count(int units, int S_max, int n_sm, bool one_k) {
     if (n_sm <= 0 || S_max < 2 * SCH) return 0;
-    if (units >= 2 * n_sm) return 1;
+    if (!one_k && units >= 2 * n_sm) return 1;
     const int want = (2 * SPLIT_CTAS * n_sm + units - 1) / units;      // about two waves of resident CTAs
     const int cap = (S_max + SCH - 1) / SCH;
     const int s = want < cap ? want : cap;
