@@ -15,6 +15,7 @@ import torch
 from oracle import sparq_oracle as O
 from paper_2312_04985_b200 import sparq
 from tests import harness as H
+from tests.test_gpu_grouped import compare_groups, run_grouped
 from tests.test_gpu_random_shapes import make
 
 pytestmark = pytest.mark.gpu
@@ -211,4 +212,8 @@ def test_random_settings(seed):
         with H.decode_plan(plan):
             gpu = run_opt(cache, q, r, k, tau_mode, realloc, window)
         compare_opt(gpu, q.numpy(), K.numpy(), V.numpy(), seq.numpy(), r, k, tau_mode, realloc, window, what + " plan=%s" % plan)
+    # the grouped selection with the same settings
+    gpu = run_grouped(cache, q, r, k, realloc=realloc, tau_mode=tau_mode, window=window)
+    compare_groups(gpu, q.numpy(), K.numpy(), V.numpy(), seq.numpy(), r, k, realloc=realloc, tau_mode=tau_mode, window=window,
+                   what=what + " grouped")
     cache.check_status(0)
