@@ -350,3 +350,27 @@ def test_step_host_with_inputs_back_to_back_in_one_buffer():
         sparq.sparq_step_host(buf, None, None, b.K, b.Kt, b.V, b.vsum, b.vbar, b.seq_lens, c.r, c.k, out_host, staging, b.status)
         np.testing.assert_array_equal(out_host.numpy().astype(np.float64), ref["out"])
     assert torch.equal(a.Kt, b.Kt) and torch.equal(a.V, b.V) and torch.equal(a.seq_lens, b.seq_lens)
+
+
+def test_largest_supported_cache_rank_and_budget():
+    """The maxima of the interface together: S_max = 262,144 positions, r = d_h = 128, k = 1024 --
+    per-head selection, the store-K-once variant, the grouped selection and a local window."""
+    from tests.test_gpu_1xk import run_1xk
+    from tests.test_gpu_grouped import compare_groups, run_grouped
+    from tests.test_gpu_opt import compare_opt, run_opt
+    S, r, k = 262144, 128, sparq.K_MAX
+    g = torch.Generator().manual_seed(77)
+    q = torch.randn(1, 2, 128, generator=g).half()
+    K = torch.randn(1, 1, S, 128, generator=g).half()
+    V = torch.randn(1, 1, S, 128, generator=g).half()
+    seq = torch.tensor([S - 5], dtype=torch.int32)
+    cache = H.DeviceCache(K, V, seq)
+    qn, Kn, Vn = q.numpy(), K.numpy(), V.numpy()
+    ora = H.oracle_all_units(qn, Kn, Vn, seq.numpy(), r, k)
+    units = (qn.reshape(2, -1), lambda u: Kn[0, 0], lambda u: Vn[0, 0], np.repeat(seq.numpy(), 2))
+    assert H.compare_units(H.flat(cache.decode(q, r, k)), ora, *units, r, k, "largest sizes") == 0
+    assert H.compare_units(H.flat(run_1xk(cache, q, r, k)), ora, *units, r, k, "largest sizes, K stored once") == 0
+    compare_groups(run_grouped(cache, q, r, k), qn, Kn, Vn, seq.numpy(), r, k, what="largest sizes, grouped")
+    gpu = run_opt(cache, q, r, k, sparq.TAU_SQRT_R, False, k // 4)
+    assert compare_opt(gpu, qn, Kn, Vn, seq.numpy(), r, k, sparq.TAU_SQRT_R, False, k // 4, "largest sizes, window") == 0
+    cache.check_status(0)
