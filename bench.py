@@ -133,15 +133,16 @@ def _sample_units(case, n_units, seed=0):
     return q, K, V, seq
 
 
-def time_oracle(case, n_units, reps=1):
-    """The C float64 oracle, as it stands, on a sample of units with every host core OpenMP gives it."""
+def time_oracle(case, n_units, reps=1, n_threads=0):
+    """The C float64 oracle, as it stands, on a sample of units with every host core OpenMP gives it
+    (n_threads = 0) or with the given number of threads."""
     from oracle import c_oracle
     q, K, V, seq = _sample_units(case, n_units)
-    cores = c_oracle.max_threads()
+    cores = c_oracle.max_threads() if n_threads == 0 else n_threads
     times = []
     for _ in range(reps):
         t0 = time.perf_counter()
-        c_oracle.sparq_decode(q, K, V, seq, case.r, case.k)
+        c_oracle.sparq_decode(q, K, V, seq, case.r, case.k, n_threads=n_threads)
         times.append(time.perf_counter() - t0)
     return len(seq), cores, times
 
@@ -457,6 +458,12 @@ def run_b200(args):
         cpu = {"value": U * reps / sum(times), "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": "%d of %d (b,h) units of %s (seeded sample), %d passes, C float64 oracle with OpenMP "
                          "over units, %.1f s in all" % (U, B * Hq, name, reps, sum(times))}
+        # the same oracle on one thread (a smaller sample: about 3 s)
+        n1 = max(1, n_sample // 16)
+        U1, _, t1 = time_oracle(case, n1, reps=1, n_threads=1)
+        reps1 = int(min(50, max(1, round(3.0 / max(t1[0], 1e-3)))))
+        U1, _, t1 = time_oracle(case, n1, reps=reps1, n_threads=1)
+        cpu["single_thread"] = {"value": U1 * reps1 / sum(t1), "unit": UNIT, "sample": "%d units, %d passes, %.1f s" % (U1, reps1, sum(t1))}
 
     traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH if (name == "c2" and args.batch is None) else None
     line = {
