@@ -297,6 +297,9 @@ def run_b200(args):
     total_ms = max_over_ranks(t_beg.elapsed_time(t_end))
     decode_ms = [ev[0].elapsed_time(ev[1]) for ev in evs if ev is not None]
     decode_us = max_over_ranks(1e3 * sum(decode_ms) / len(decode_ms))
+    # standard error of that mean over the sampled launches (this rank's)
+    _m = sum(decode_ms) / len(decode_ms)
+    decode_us_stderr = 1e3 * (sum((x - _m) ** 2 for x in decode_ms) / max(1, len(decode_ms) - 1)) ** 0.5 / len(decode_ms) ** 0.5
     if int(status.item()) != 0:
         raise SystemExit("device status %s" % sparq.status_string(int(status.item())))
     us_per_step = 1e3 * total_ms / args.steps
@@ -478,7 +481,8 @@ def run_b200(args):
                          % ("inputs larger than L2" if n_copies == 1 else "steps rotate over independent cache copies larger than L2 together",
                             cache_bytes / 1e9, n_copies, "y" if n_copies == 1 else "ies", POOL),
                    "parallelism": "independent batches per GPU, no collective"},
-        "us_per_step": us_per_step, "graph_replay_us_per_step": graph_us, "sparq_decode_us": decode_us, "sparq_decode_full_len_us": sparq_full_us,
+        "us_per_step": us_per_step, "graph_replay_us_per_step": graph_us, "sparq_decode_us": decode_us, "sparq_decode_us_stderr": decode_us_stderr,
+        "sparq_decode_launches_timed": len(decode_ms), "sparq_decode_full_len_us": sparq_full_us,
         "dense_decode_us": dense_us, "speedup_vs_dense": dense_us / sparq_full_us, "sparq_decode_grouped": grouped,
         "sparq_decode_1xk": one_k, "sparq_decode_opt_window": windowed,
         "dense_hbm_gbs": dense_bytes(B, Hq, Hkv, end_mean, d) / (dense_us * 1e-6) / 1e9,
