@@ -6,7 +6,7 @@ import subprocess
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
-SOURCES = [os.path.join(_PKG, "csrc", f) for f in ("api.cu", "sparq_decode.cu", "sparq_decode_pipe.cu", "sparq_decode_grouped.cu",
+SOURCES = [os.path.join(_PKG, "csrc", f) for f in ("api.cu", "sparq_decode.cu", "sparq_decode_pipe.cu", "sparq_decode_wide.cu", "sparq_decode_grouped.cu",
                                                      "dense_decode.cu", "cache.cu")]
 HEADERS = [os.path.join(_ROOT, "include", "sparq.h")] + [os.path.join(_PKG, "csrc", f)
                                                         for f in ("common.cuh", "decode_common.cuh", "kernels.h")]

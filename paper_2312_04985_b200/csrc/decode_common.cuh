@@ -200,6 +200,54 @@ __device__ __forceinline__ uint32_t group_scan_incl(uint32_t v, uint32_t* red, u
     return v + before;
 }
 
+// Stage a1 by a whole CTA (G::NT >= 128 threads): the r largest |q_j| by rank counting.
+// key = |q_j| bit pattern above (127 - j): distinct keys, larger |q| first, then smaller j.
+// Fills hm.qf, q16, i1 (ascending), qh (zero padded to a multiple of RB_), inv_tau, l1_sel.
+// red: 2*NW floats, cnt: 4 words.  Ends with a barrier.
+template <class G, int RB_>
+__device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restrict__ q_row, int r, HeadMeta& hm, float* red,
+                                            uint32_t* cnt, uint32_t opts) {
+    const int lane = tid & 31, warp = tid >> 5;
+    uint16_t hb = 0;
+    float qf = 0.f, aq = 0.f;
+    uint32_t mine = 0;
+    if (tid < D) {
+        hb = q_row[tid];
+        qf = __half2float(__ushort_as_half(hb));
+        aq = fabsf(qf);
+        mine = ((uint32_t)(hb & 0x7fffu) << 7) | (uint32_t)(D - 1 - tid);
+        hm.qf[tid] = qf;
+        hm.q16[tid] = hb;
+        hm.rkey[tid] = mine;
+    }
+    G::sync();
+    bool sel = false;
+    if (tid < D) {
+        int rank = 0;
+        const uint4* rk4 = reinterpret_cast<const uint4*>(hm.rkey);
+#pragma unroll 8
+        for (int j = 0; j < D / 4; ++j) {
+            uint4 o = rk4[j];
+            rank += (o.x > mine) + (o.y > mine) + (o.z > mine) + (o.w > mine);
+        }
+        sel = rank < r;
+    }
+    const unsigned bal = __ballot_sync(FULL, sel);
+    if (lane == 0 && warp < 4) cnt[warp] = __popc(bal);      // warps 0..3 hold the D components
+    float l1_all = aq, l1_sel = sel ? aq : 0.f;
+    group_sum2<G>(l1_all, l1_sel, red, tid);                 // its barriers also publish cnt
+    if (sel) {
+        int slot = __popc(bal & ((1u << lane) - 1));
+        for (int w = 0; w < warp; ++w) slot += cnt[w];
+        hm.i1[slot] = tid;                                   // ascending by construction
+        hm.qh[slot] = hb;
+    }
+    const int r_pad = (r + RB_ - 1) / RB_ * RB_;
+    if (tid >= r && tid < r_pad) hm.qh[tid] = 0;
+    if (tid == 0) { hm.inv_tau = opt_inv_tau(opts, l1_all, l1_sel, r); hm.l1_sel = l1_sel; }
+    G::sync();
+}
+
 // One radix-select pass over an already filled histogram: find, from the top, the bin holding the
 // need-th largest candidate.  res[0] = bin, res[1] = candidates above it, res[2] = candidates in
 // it.  All threads of the group call; the result is valid after the trailing barrier.

@@ -38,11 +38,11 @@ def test_c0_tiny_single_step_against_numpy_oracle():
     _dense_check(c, cache, c.q_steps[0], "c0")
 
 
-@pytest.mark.parametrize("plan", ["split", "pipe", "simple"])
+@pytest.mark.parametrize("plan", ["split", "pipe", "simple", "wide"])
 def test_c1_llama2_batch1_all_heads(plan):
     """Batch 1, 32 heads: fewer units than SMs.  The library's own choice at this length is the
-    persistent kernel (one CTA per unit); the sliced plan and the one-CTA-per-unit kernel must give
-    the same parity."""
+    wide kernel (one 512-thread CTA per unit); the sliced plan, the persistent kernel and the
+    one-CTA-per-unit kernel must give the same parity."""
     c = synth.make_case("c1")
     with H.decode_plan(plan):
         assert (sparq.sparq_workspace_bytes(1, 32, 32, 128, 4096, 32, 128) > 0) == (plan == "split")
@@ -60,7 +60,7 @@ def test_split_plan_long_ragged_gqa_and_bad_length():
     assert total == 24 and waived <= 1
     cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
     q = c.q_steps[0]
-    a = cache.decode(q, c.r, c.k)                                   # library's choice: split (24 units)
+    a = cache.decode(q, c.r, c.k)                                   # library's choice: the wide kernel (24 units)
     with H.decode_plan("simple"):
         b = cache.decode(q, c.r, c.k)
     np.testing.assert_array_equal(a["i1"], b["i1"])
