@@ -37,7 +37,7 @@ L2_BYTES = 126e6
 EV_EVERY = 4          # steps between CUDA-event pairs around the decode inside the timed region
 # which decode kernel the library picks per workload (caches too long for the persistent kernel's
 # shared memory take the split-plan kernel); every step launches the append kernel and one decode kernel
-DECODE_KERNEL = {"c1": "sparq_decode_wide_kernel", "c3": "sparq_split_kernel", "c4": "sparq_decode_wide_kernel"}
+DECODE_KERNEL = {"c1": "sparq_decode_wide_kernel", "c3": "sparq_decode_wide_kernel", "c4": "sparq_decode_wide_kernel"}
 LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,

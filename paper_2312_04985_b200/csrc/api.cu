@@ -28,10 +28,11 @@ int device_sm_count() {
 }
 
 // SPARQ_DECODE_PLAN=simple|pipe|split|wide forces one of the sparq_decode plans (tests and tuning).
-// Unset or anything else: the wide kernel (one 512-thread CTA per unit) for up to one unit per SM
-// and, on caches too long for the persistent kernel, for up to four units per SM or units with
-// 2 MB or more to stream; the persistent pipelined kernel wherever else one unit's keys fit its
-// shared memory; otherwise the split plan if the caller passed its workspace; else one CTA per unit.
+// Unset or anything else: the wide kernel (one CTA of 512 threads, or two of 256, per SM; a unit's
+// keys in shared memory) for up to one unit per SM and for caches too long for the persistent
+// kernel; the persistent pipelined kernel wherever else one unit's keys fit its shared memory;
+// beyond the wide kernel's reach (about 44,000 positions) the split plan if the caller passed its
+// workspace; else one CTA per unit.
 int forced_plan() {
     const char* e = getenv("SPARQ_DECODE_PLAN");
     if (!e) return 0;
@@ -109,18 +110,24 @@ static bool split_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok)
     return units < n_sm && (size_t)2 * S_max * r > ((size_t)512 << 10);
 }
 
-// The wide kernel (one 512-thread CTA per unit, nothing overlapping one unit with the next) against
-// the others, where its keys fit in shared memory.  Up to one unit per SM it is the fastest at any
-// length (32 units of 4096 positions: 19.8 us, persistent kernel 22.7, sliced plan 27.6; 128 units
-// of 16384 at r = 16: 28.6 against the sliced plan's 58.2).  Beyond that the persistent kernel wins
-// wherever it fits (160 units of 4096: 28.5 against 32.4 us).  Against the split plan on longer
-// caches it wins up to about four units per SM (256 units of 16384, r = 16: 48.7 against 71.3 us;
-// 512: equal; 768 and 1024: 5 % slower) and at any count when a unit has a lot to stream (512 units
-// of up to 32800 positions at r = 64: 260 against 289 us).
-static bool wide_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok) {
-    if (units <= n_sm) return true;
-    if (pipe_ok) return false;
-    return units <= 4 * n_sm || (size_t)2 * S_max * r >= ((size_t)2 << 20);
+// The wide kernel against the others, where its keys fit in shared memory.  Up to one unit per SM it
+// is the fastest at any length (32 units of 4096 positions: 19.8 us, persistent kernel 22.7, sliced
+// plan 27.6; 128 units of 16384 at r = 16: 28.6 against the sliced plan's 58.2).  Beyond that the
+// persistent kernel wins wherever it fits (2048 units of 4096: 128 against 161 us), and the wide
+// kernel wins on the longer caches (1024 units of 16384, r = 16, two CTAs per SM: 141 against the
+// split plan's 147 us; 256 units: 43 against 71; 512 units of up to 32800 positions at r = 64, one
+// CTA per SM: 260 against 289).
+static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= n_sm || !pipe_ok; }
+
+// Two 256-thread CTAs per SM instead of one of 512 threads: with more units than SMs, where both fit.
+// SPARQ_WIDE_PAIRS=0|1 overrides (tuning).
+static bool wide_pairs(int units, int S_max, int n_sm) {
+    int dev = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+        return false;
+    bool pairs = units > n_sm && wide_pair_fits(S_max, per_sm);
+    if (const char* e = getenv("SPARQ_WIDE_PAIRS")) pairs = (e[0] == '1') && wide_pair_fits(S_max, per_sm);
+    return pairs;
 }
 
 size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, int k) {
@@ -130,7 +137,7 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     const int splits = S_max <= SPARQ_S_MAX_WORKSPACE ? split_count(B * Hq, S_max, n_sm) : 0;
     const bool pipe_ok = pipe_fits(S_max, device_smem_optin());
     const int plan = forced_plan();                          // a plan forced through the environment gets what it needs
-    if (plan == 4 || (plan == 0 && wide_fits(S_max, device_smem_optin()) && wide_preferred(B * Hq, S_max, r, n_sm, pipe_ok)))
+    if (plan == 4 || (plan == 0 && wide_fits(S_max, device_smem_optin()) && wide_preferred(B * Hq, n_sm, pipe_ok)))
         return 0;
     if (splits && (plan == 3 || (plan == 0 && split_preferred(B * Hq, S_max, r, n_sm, pipe_ok))))
         return split_scratch_bytes(B * Hq, S_max, splits);
@@ -160,9 +167,9 @@ static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_hal
     // their length, and beside the split plan for caches the persistent kernel cannot hold
     const bool wide_ok = wide_fits(S_max, device_smem_optin());
     if (plan == 4 && !wide_ok) return SPARQ_ERR_TOO_LONG;
-    if (wide_ok && (plan == 4 || (plan == 0 && wide_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin())))))
+    if (wide_ok && (plan == 4 || (plan == 0 && wide_preferred(B * Hq, n_sm, pipe_fits(S_max, device_smem_optin())))))
         return rc(launch_sparq_decode_wide(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha,
-                                           status, (cudaStream_t)stream));
+                                           status, wide_pairs(B * Hq, S_max, n_sm), (cudaStream_t)stream));
     const bool split_pays = split_preferred(B * Hq, S_max, r, n_sm, pipe_fits(S_max, device_smem_optin()));
     if (ws_ok && (plan == 3 || (plan == 0 && split_pays)))
         return rc(launch_sparq_decode_split(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,

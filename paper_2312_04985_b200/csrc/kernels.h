@@ -43,10 +43,11 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
 
 // sparq_decode_wide.cu: one CTA of 512 threads per unit, for a handful of units (batch-1 latency)
 bool wide_fits(int S_max, int smem_optin);
+bool wide_pair_fits(int S_max, int smem_per_sm);
 cudaError_t launch_sparq_decode_wide(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, cudaStream_t stream);
+                                     int32_t* status, bool pairs, cudaStream_t stream);
 
 // sparq_decode_grouped.cu: group-shared selection (one CTA per KV head)
 int grouped_slices(int groups, int S_max, int n_sm);

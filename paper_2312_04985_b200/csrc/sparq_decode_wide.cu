@@ -18,16 +18,14 @@
 namespace sparq {
 namespace {
 
-constexpr int WNT = 512;
-constexpr int WCH = WNT * 8;             // positions per pass: a vector of 8 per thread
 constexpr int WROWS = 16;                // Kt rows in flight per thread
-using WCTA = Group<WNT, 0>;
 
+template <int WNT>
 struct WideShared {
     HeadMeta hm;
     int32_t i2[SPARQ_K_MAX];
-    float red[2 * WCTA::NW];
-    uint32_t redu[2 * WCTA::NW];
+    float red[2 * (WNT / 32)];
+    uint32_t redu[2 * (WNT / 32)];
     uint32_t res[4];
     uint32_t band[4];
     uint32_t cnt[4];
@@ -36,7 +34,10 @@ struct WideShared {
 __host__ __device__ constexpr int wide_bm_words(int S_max) { return (S_max + 127) / 128 * 4; }
 __host__ __device__ constexpr size_t wide_keys_bytes(int S_max) { return ((size_t)S_max * 4 + 127) & ~(size_t)127; }
 
-__global__ void __launch_bounds__(WNT, 1)
+// WNT = 512: one CTA per SM (the latency form).  WNT = 256: two CTAs per SM where their keys fit, so that
+// one unit's select and gather overlap another's stream (many units on a long cache).
+template <int WNT>
+__global__ void __launch_bounds__(WNT, WNT == 512 ? 1 : 2)
 sparq_decode_wide_kernel(const sparq_half* __restrict__ q, const sparq_half* __restrict__ K,
                          const sparq_half* __restrict__ Kt, const sparq_half* __restrict__ V,
                          const sparq_half* __restrict__ vbar, const int32_t* __restrict__ seq_lens,
@@ -47,7 +48,9 @@ sparq_decode_wide_kernel(const sparq_half* __restrict__ q, const sparq_half* __r
     uint32_t* keys = reinterpret_cast<uint32_t*>(dyn_smem);                           // [S_max] approximate-score keys
     uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn_smem + wide_keys_bytes(S_max));  // [FBINS] histogram of the keys' top bits
     unsigned char* scratch = reinterpret_cast<unsigned char*>(hist1 + FBINS);         // the post phase's scratch
-    __shared__ WideShared sh;
+    using WCTA = Group<WNT, 0>;
+    constexpr int WCH = WNT * 8;                             // positions per pass: a vector of 8 per thread
+    __shared__ WideShared<WNT> sh;
     HeadMeta& hm = sh.hm;
 
     const int tid = threadIdx.x;
@@ -141,26 +144,31 @@ sparq_decode_wide_kernel(const sparq_half* __restrict__ q, const sparq_half* __r
                     true, opt_realloc(opts));
 }
 
-size_t wide_dynamic_smem(int S_max) {
+size_t wide_dynamic_smem(int S_max, int nt) {
     return wide_keys_bytes(S_max) + (size_t)FBINS * 4 +
-           ((post_scratch_bytes(WCTA::NHW, wide_bm_words(S_max)) + 127) & ~(size_t)127);
+           ((post_scratch_bytes(nt / 16, wide_bm_words(S_max)) + 127) & ~(size_t)127);
 }
 
 }  // namespace
 
 bool wide_fits(int S_max, int smem_optin) {
-    return wide_dynamic_smem(S_max) + sizeof(WideShared) + 1024 <= (size_t)smem_optin;
+    return wide_dynamic_smem(S_max, 512) + sizeof(WideShared<512>) + 1024 <= (size_t)smem_optin;
+}
+// two 256-thread CTAs of this S_max per SM (each CTA also costs 1 KB of the SM's shared memory)
+bool wide_pair_fits(int S_max, int smem_per_sm) {
+    return 2 * (wide_dynamic_smem(S_max, 256) + sizeof(WideShared<256>) + 1024) <= (size_t)smem_per_sm;
 }
 
 cudaError_t launch_sparq_decode_wide(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, cudaStream_t stream) {
-    const size_t dyn = wide_dynamic_smem(S_max);
-    cudaError_t e = cudaFuncSetAttribute(sparq_decode_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+                                     int32_t* status, bool pairs, cudaStream_t stream) {
+    const int nt = pairs ? 256 : 512;
+    const size_t dyn = wide_dynamic_smem(S_max, nt);
+    auto kernel = pairs ? sparq_decode_wide_kernel<256> : sparq_decode_wide_kernel<512>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
-    sparq_decode_wide_kernel<<<B * Hq, WNT, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, opts, out, idx_r,
-                                                            idx_k, alpha, status);
+    kernel<<<B * Hq, nt, dyn, stream>>>(q, K, Kt, V, vbar, seq_lens, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha, status);
     return cudaGetLastError();
 }
 
