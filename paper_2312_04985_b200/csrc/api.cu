@@ -76,12 +76,30 @@ const char* sparq_status_string(int code) {
     }
 }
 
-int sparq_max_seq_len(void) {
+// largest S_max of the one-CTA-per-unit kernel with the bulk-copy ring (a forced plan "simple")
+static int simple_max_seq_len() {
     long avail = (long)device_smem_optin() - (long)decode_static_smem() - (long)decode_dynamic_smem(0) - 1024;
     if (avail <= 0) return 0;
     long s = (avail / 4) & ~7L;
     long cap = decode_max_positions();
     return (int)(s < cap ? s : cap);
+}
+
+// largest S_max of the wide kernel: its shared memory grows with S_max, so bisect on multiples of 8
+static int wide_max_seq_len() {
+    const int optin = device_smem_optin();
+    int lo = 0, hi = SPARQ_S_MAX_WORKSPACE / 8;              // in units of 8 positions; lo fits (or is 0), hi may not
+    if (wide_fits(hi * 8, optin)) return hi * 8;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) / 2;
+        if (wide_fits(mid * 8, optin)) lo = mid; else hi = mid;
+    }
+    return lo * 8;
+}
+
+int sparq_max_seq_len(void) {
+    const int a = simple_max_seq_len(), b = wide_max_seq_len();
+    return a > b ? a : b;
 }
 
 int sparq_cache_build(const sparq_half* K, const sparq_half* V, const int32_t* seq_lens,
@@ -177,6 +195,7 @@ static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_hal
     if (too_long) return SPARQ_ERR_TOO_LONG;                 // a plan without scratch was forced
     const bool fits = pipe_fits(S_max, device_smem_optin());
     if (plan == 2 && !fits) return SPARQ_ERR_TOO_LONG;
+    if (plan == 1 && S_max > simple_max_seq_len()) return SPARQ_ERR_TOO_LONG;
     if (fits && plan != 1) {
         // with a workspace the persistent CTAs draw their units from a counter instead of a fixed share
         unsigned int* counter = (workspace && workspace_bytes >= SPARQ_PIPE_WORKSPACE_BYTES && B * Hq > n_sm)
