@@ -36,13 +36,17 @@ POOL = 16            # distinct (q, k_new, v_new) sets rotated through the steps
 L2_BYTES = 126e6
 EV_EVERY = 4          # steps between CUDA-event pairs around the decode inside the timed region
 # which decode kernel the library picks per workload (caches too long for the persistent kernel's
-# shared memory take the split-plan kernel); every step launches the append kernel and one decode kernel
+# shared memory take the wide kernel); every step launches the append kernel and one decode kernel
 DECODE_KERNEL = {"c1": "sparq_decode_wide_kernel", "c3": "sparq_decode_wide_kernel", "c4": "sparq_decode_wide_kernel"}
 LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 681.0e6   # 2 x (336.49 + 4.02) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    "c2": 681.0e6,   # 2 x (336.47 + 4.05) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md (B = 32 capture, scaled by the units)
+    "c3": 508.5e6,   # 505.1 + 3.4 MB: profiles/sparq_decode_wide_kernel_c3_c4.md
+    "c4": 812.5e6,   # 808.8 + 3.7 MB: the same file (the heads of a group share rows in the L2)
+}
 
 
 def compulsory_bytes_per_unit(n: float, r: int, k: int, d: int) -> float:
@@ -468,7 +472,7 @@ def run_b200(args):
         U1, _, t1 = time_oracle(case, n1, reps=reps1, n_threads=1)
         cpu["single_thread"] = {"value": U1 * reps1 / sum(t1), "unit": UNIT, "sample": "%d units, %d passes, %.1f s" % (U1, reps1, sum(t1))}
 
-    traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH if (name == "c2" and args.batch is None) else None
+    traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name) if args.batch is None else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": us_per_step / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
