@@ -374,3 +374,36 @@ def test_largest_supported_cache_rank_and_budget():
     gpu = run_opt(cache, q, r, k, sparq.TAU_SQRT_R, False, k // 4)
     assert compare_opt(gpu, qn, Kn, Vn, seq.numpy(), r, k, sparq.TAU_SQRT_R, False, k // 4, "largest sizes, window") == 0
     cache.check_status(0)
+
+
+def test_longest_cache_without_workspace():
+    """S_max = sparq_max_seq_len(): the longest cache whose approximate scores still fit in shared
+    memory (no workspace passed), at the largest rank and budget."""
+    S = sparq.sparq_max_seq_len()
+    assert S % 8 == 0 and 40000 < S < 65536
+    r, k = 128, sparq.K_MAX
+    g = torch.Generator().manual_seed(78)
+    q = torch.randn(1, 2, 128, generator=g).half()
+    K = torch.randn(1, 1, S, 128, generator=g).half()
+    V = torch.randn(1, 1, S, 128, generator=g).half()
+    seq = torch.tensor([S - 3], dtype=torch.int32)
+    cache = H.DeviceCache(K, V, seq)
+    qd = q.cuda()
+    out = torch.empty_like(qd)
+    idx_r = torch.empty(1, 2, r, dtype=torch.int32, device="cuda")
+    idx_k = torch.empty(1, 2, k, dtype=torch.int32, device="cuda")
+    alpha = torch.empty(1, 2, dtype=torch.float32, device="cuda")
+    sparq.sparq_decode(qd, cache.K, cache.Kt, cache.V, cache.vbar, cache.seq_lens, r, k, out, idx_r=idx_r, idx_k=idx_k,
+                       alpha=alpha, workspace=None, status=cache.status)
+    gpu = dict(out=out.cpu().numpy().astype(np.float64), i1=idx_r.cpu().numpy(), i2=idx_k.cpu().numpy(),
+               alpha=alpha.cpu().numpy().astype(np.float64))
+    qn, Kn, Vn = q.numpy(), K.numpy(), V.numpy()
+    ora = H.oracle_all_units(qn, Kn, Vn, seq.numpy(), r, k)
+    assert H.compare_units(H.flat(gpu), ora, qn.reshape(2, -1), lambda u: Kn[0, 0], lambda u: Vn[0, 0],
+                           np.repeat(seq.numpy(), 2), r, k, "longest without workspace") == 0
+    with pytest.raises(sparq.SparqError) as e:                 # eight positions more need the workspace
+        big = torch.zeros(1, 1, S + 8, 128, dtype=torch.float16, device="cuda")
+        sparq.sparq_decode(qd, big, torch.zeros(1, 1, 128, S + 8, dtype=torch.float16, device="cuda"), big,
+                           cache.vbar, cache.seq_lens, r, k, out)
+    assert e.value.code == sparq.ERR_WORKSPACE
+    cache.check_status(0)
