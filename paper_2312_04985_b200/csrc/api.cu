@@ -121,8 +121,9 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
                                   (cudaStream_t)stream));
 }
 
-// Which plan pays: the persistent kernel wherever one unit's keys fit its shared memory, except for
-// a few units (fewer than SMs) with a lot to stream each, which the split plan slices over all SMs.
+// The split plan against the persistent kernel where the wide kernel does not apply (a forced plan,
+// or a cache beyond the wide kernel's shared memory): wherever the persistent kernel does not fit,
+// and for a few units (fewer than SMs) with a lot to stream each, which it slices over all SMs.
 static bool split_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok) {
     if (!pipe_ok) return true;
     return units < n_sm && (size_t)2 * S_max * r > ((size_t)512 << 10);

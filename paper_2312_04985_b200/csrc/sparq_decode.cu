@@ -1,6 +1,8 @@
-// sparq_decode, one CTA per (batch, query head): the kernel for long sequences (any S_max whose
-// score keys fit in shared memory).  Every stage is fused so that only the compulsory bytes touch
-// HBM.
+// sparq_decode, one CTA per (batch, query head) fed by a ring of bulk copies (any S_max whose score
+// keys fit in shared memory beside the ring), and -- further down -- the split plan for caches
+// beyond shared memory.  Every stage is fused so that only the compulsory bytes touch HBM.  (The
+// ring kernel runs only when forced: the wide kernel of sparq_decode_wide.cu is faster at every
+// shape; it stays as an independent implementation for the tests to compare the others with.)
 //
 //   a1  top-r of |q| by rank counting on integer keys; tau                    (Step 1, Eq. (9))
 //   a2  stream the r selected rows of Kt through a ring of bulk asynchronous copies

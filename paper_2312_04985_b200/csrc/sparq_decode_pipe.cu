@@ -8,7 +8,7 @@
 //                     alternate stages and lanes issue one row each, because one thread (and even
 //                     one warp) can only start a copy every few hundred cycles
 //   stream group      a2: consumes the ring, fp32 mixed-precision FMA chain per position, writes the
-//                     order-preserving keys of unit j into key buffer j mod 3
+//                     order-preserving keys of unit j into key buffer j mod NKB (4 where they fit, else 3)
 //   post groups 0/1   a3-a6 of units j = 0,2,4,.. / 1,3,5,.. (decode_common.cuh): radix select with
 //                     exact re-decision of the threshold band, alpha, K/V row gather, combine
 //
