@@ -3,29 +3,45 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "kernels.h"
+
+namespace sparq {
+
+// The current device's figures the plan selection needs, queried once per device: the attribute
+// queries cost more than the rest of a call's host work (batch-1 decoding is host-bound without
+// CUDA graphs).  Zeros when there is no device (the host-side checks still work).
+DeviceInfo device_info() {
+    constexpr int kMax = 64;
+    static DeviceInfo table[kMax];
+    static std::atomic<int> ready[kMax];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DeviceInfo{0, 0, 0};
+    const bool cached = dev >= 0 && dev < kMax;
+    if (cached && ready[dev].load(std::memory_order_acquire)) return table[dev];
+    DeviceInfo d{0, 0, 0};
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+        return DeviceInfo{0, 0, 0};
+    if (cached) { table[dev] = d; ready[dev].store(1, std::memory_order_release); }   // (racing threads store the same values)
+    return d;
+}
+
+}  // namespace sparq
 
 namespace {
 
 using namespace sparq;
 
-int device_smem_optin() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
-    return v;
-}
+int device_smem_optin() { return device_info().smem_optin; }
 
 bool bad_common(int B, int Hq, int Hkv, int d, int S_max) {
     return B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || d != SPARQ_HEAD_DIM || S_max < 8 || S_max % 8 != 0;
 }
 
-int device_sm_count() {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-    return v;
-}
+int device_sm_count() { return device_info().sm_count; }
 
 // SPARQ_DECODE_PLAN=simple|pipe|split|wide forces one of the sparq_decode plans (tests and tuning).
 // Unset or anything else: the wide kernel (one CTA of 512 threads, or two of 256, per SM; a unit's
@@ -141,9 +157,8 @@ static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= 
 // Two 256-thread CTAs per SM instead of one of 512 threads: with more units than SMs, where both fit.
 // SPARQ_WIDE_PAIRS=0|1 overrides (tuning).
 static bool wide_pairs(int units, int S_max, int n_sm) {
-    int dev = 0, per_sm = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
-        return false;
+    const int per_sm = device_info().smem_per_sm;
+    if (per_sm <= 0) return false;
     bool pairs = units > n_sm && wide_pair_fits(S_max, per_sm);
     if (const char* e = getenv("SPARQ_WIDE_PAIRS")) pairs = (e[0] == '1') && wide_pair_fits(S_max, per_sm);
     return pairs;

@@ -8,6 +8,11 @@
 
 namespace sparq {
 
+// api.cu: multiprocessors, largest opt-in shared memory per block, shared memory per multiprocessor of
+// the current device (cached per device; zeros without a device)
+struct DeviceInfo { int sm_count, smem_optin, smem_per_sm; };
+DeviceInfo device_info();
+
 // `opts` of the decode launchers: the call's settings in one word (0 = Eq. (9) temperature, Step 3
 // applied, no local window).  Bits 0-1: temperature (SPARQ_TAU_*), bit 2: Step 3 left out,
 // bits 16-31: local window.

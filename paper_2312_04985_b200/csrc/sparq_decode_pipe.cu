@@ -478,9 +478,7 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
     a.q = q; a.K = K; a.Kt = Kt; a.V = V; a.vbar = vbar; a.seq_lens = seq_lens;
     a.n_units = B * Hq; a.Hq = Hq; a.Hkv = Hkv; a.S_max = S_max; a.S_cap = pipe_s_cap(S_max); a.r = r; a.k = k;
     a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status; a.unit_counter = unit_counter;
-    int dev = 0, smem_optin = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    const int smem_optin = device_info().smem_optin;
     const bool four = pipe_fits_nkb(S_max, smem_optin, 4);
     const size_t dyn = pipe_dynamic_smem(a.S_cap, four ? 4 : 3);
     auto kernel = opts ? (four ? sparq_decode_pipe_kernel<4, true> : sparq_decode_pipe_kernel<3, true>)
