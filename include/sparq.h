@@ -173,7 +173,9 @@ int sparq_decode_opt(const sparq_half* q, const sparq_half* K, const sparq_half*
 /*
  * dense_decode -- dense decode attention, Eq. (2), over the n = seq_lens[b] valid positions:
  * the comparison kernel for the speed-up figure (Section 6.1, "Dense" baseline).  One pass
- * over K and V per KV head serves all Hq/Hkv query heads of its group.  The sequence is split
+ * over K and V per KV head serves all Hq/Hkv query heads of its group (eight, four, two or one
+ * at a time; eight and four on the tensor cores, the softmax weights rounded to fp16 for the
+ * second product).  The sequence is split
  * across thread blocks; partial softmax states go through `workspace`
  * (dense_workspace_bytes(); contents undefined afterwards).
  */

@@ -1,8 +1,10 @@
 // dense_decode: dense single-token decode attention, Eq. (2), the comparison kernel for the
 // speed-up figure.  One CTA per (split, KV head, batch): a CTA covers one slice of the sequence of one KV head
-// for all (up to 8 at a time) query heads of its group, so K and V are read once per KV head;
-// half-warp per cache row, 128-bit loads, online softmax in fp32.  With more than one split the
-// per-split softmax states go through a scratch buffer and a small merge kernel.
+// for all (up to 8 at a time) query heads of its group, so K and V are read once per KV head.
+// One or two heads at a time: half-warp per cache row, 128-bit loads, online softmax in fp32, on the
+// CUDA cores.  Four or eight at a time: the pass is a small dense contraction and runs on the tensor
+// cores (further down).  With more than one split the per-split softmax states go through a scratch
+// buffer and a small merge kernel.
 #include <mutex>
 
 #include "common.cuh"

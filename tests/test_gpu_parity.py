@@ -407,3 +407,28 @@ def test_longest_cache_without_workspace():
                            cache.vbar, cache.seq_lens, r, k, out)
     assert e.value.code == sparq.ERR_WORKSPACE
     cache.check_status(0)
+
+
+@pytest.mark.parametrize("g", [1, 2, 3, 4, 5, 8, 12])
+def test_dense_decode_group_sizes(g):
+    """dense_decode serves a KV head's query heads eight, four, two or one at a time (eight and four on
+    the tensor cores): every mix of those passes, ragged lengths with tiles that end inside their 16
+    positions, one position only, and the split and unsplit plans -- against the float64 oracle; a bad
+    length among the sequences gives a zero row and the status."""
+    gen = torch.Generator().manual_seed(100 + g)
+    for B, Hkv, S, lens in ((3, 2, 1056, [1056, 517, 1]), (40, 4, 272, None)):
+        Hq = Hkv * g
+        q = torch.randn(B, Hq, 128, generator=gen).half()
+        K = torch.randn(B, Hkv, S, 128, generator=gen).half()
+        V = torch.randn(B, Hkv, S, 128, generator=gen).half()
+        seq = torch.tensor(lens if lens else torch.randint(1, S + 1, (B,), generator=gen).tolist(), dtype=torch.int32)
+        cache = H.DeviceCache(K, V, seq, poison=True)
+        got = cache.dense(q)
+        want = c_oracle.dense_decode(q.numpy(), K.numpy(), V.numpy(), seq.numpy())
+        H.check_out(got.reshape(want.shape), want, "dense g=%d B=%d" % (g, B))
+        cache.check_status(0)
+    cache.seq_lens[1] = 0
+    bad = cache.dense(q)
+    cache.check_status(sparq.DEV_BAD_SEQ_LEN)
+    assert (bad[1] == 0).all()
+    np.testing.assert_array_equal(bad[0], got[0])
