@@ -56,10 +56,12 @@ int forced_plan() {
     if (!strcmp(e, "pipe")) return 2;
     if (!strcmp(e, "split")) return 3;
     if (!strcmp(e, "wide")) return 4;
+    if (!strcmp(e, "pipe16")) return 5;
     return 0;
 }
 
 constexpr size_t SPARQ_PIPE_WORKSPACE_BYTES = 64;
+static size_t pipe_split_bytes(int S_max, int n_sm) { return pipe_split_workspace(S_max, n_sm); }
 
 int rc(cudaError_t e) { return e == cudaSuccess ? SPARQ_OK : SPARQ_ERR_CUDA; }
 
@@ -171,6 +173,7 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     const int splits = S_max <= SPARQ_S_MAX_WORKSPACE ? split_count(B * Hq, S_max, n_sm) : 0;
     const bool pipe_ok = pipe_fits(S_max, device_smem_optin());
     const int plan = forced_plan();                          // a plan forced through the environment gets what it needs
+    if (plan == 5) return pipe_split_fits(S_max, device_smem_optin()) ? pipe_split_bytes(S_max, n_sm) : 0;
     if (plan == 4 || (plan == 0 && wide_fits(S_max, device_smem_optin()) && wide_preferred(B * Hq, n_sm, pipe_ok)))
         return 0;
     if (splits && (plan == 3 || (plan == 0 && split_preferred(B * Hq, S_max, r, n_sm, pipe_ok))))
@@ -199,6 +202,13 @@ static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_hal
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
     // one 512-thread CTA per unit with the keys in shared memory: the choice for a handful of units whatever
     // their length, and beside the split plan for caches the persistent kernel cannot hold
+    if (plan == 5) {
+        if (!pipe_split_fits(S_max, device_smem_optin())) return SPARQ_ERR_TOO_LONG;
+        if (!workspace || workspace_bytes < pipe_split_bytes(S_max, n_sm)) return SPARQ_ERR_WORKSPACE;
+        return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
+                                           alpha, status, n_sm, static_cast<unsigned int*>(workspace), true,
+                                           (cudaStream_t)stream));
+    }
     const bool wide_ok = wide_fits(S_max, device_smem_optin());
     if (plan == 4 && !wide_ok) return SPARQ_ERR_TOO_LONG;
     if (wide_ok && (plan == 4 || (plan == 0 && wide_preferred(B * Hq, n_sm, pipe_fits(S_max, device_smem_optin())))))
@@ -217,7 +227,7 @@ static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_hal
         unsigned int* counter = (workspace && workspace_bytes >= SPARQ_PIPE_WORKSPACE_BYTES && B * Hq > n_sm)
                                     ? static_cast<unsigned int*>(workspace) : nullptr;
         return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
-                                           alpha, status, n_sm, counter, (cudaStream_t)stream));
+                                           alpha, status, n_sm, counter, false, (cudaStream_t)stream));
     }
     return rc(launch_sparq_decode(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k, alpha,
                                   status, (cudaStream_t)stream));

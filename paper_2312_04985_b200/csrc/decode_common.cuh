@@ -307,6 +307,23 @@ static __device__ __noinline__ double dot64_at_batched(const sparq_half* Kt_head
     return acc;
 }
 
+// The approximate-score keys of a unit as the post stages see them: one array of 32-bit keys, or the
+// keys' upper halves in one array (shared memory) and their lower halves in another (global memory,
+// read around the L1).  key_coarse: the key with at least its upper 16 bits right and the rest zero or
+// right -- enough for the first digit; key_full: all 32 bits.
+struct SplitKeys {
+    const uint16_t* hi;
+    const uint16_t* lo;
+};
+__device__ __forceinline__ uint32_t key_full(const uint32_t* keys, int t) { return keys[t]; }
+__device__ __forceinline__ uint32_t key_coarse(const uint32_t* keys, int t) { return keys[t]; }
+__device__ __forceinline__ uint32_t key_coarse(SplitKeys keys, int t) { return (uint32_t)keys.hi[t] << 16; }
+__device__ __forceinline__ uint32_t key_full(SplitKeys keys, int t) {
+    return ((uint32_t)keys.hi[t] << 16) | (uint32_t)__ldcg(keys.lo + t);
+}
+template <class T> struct keys_split { static constexpr bool value = false; };
+template <> struct keys_split<SplitKeys> { static constexpr bool value = true; };
+
 // What a select variant hands to finish(): the selection bitmap sc.bm_sel (and, in the degenerate
 // path, the tie bitmap sc.bm_tie with need_tie of its lowest positions wanted) and the softmax
 // denominator of the approximate scores relative to the largest key.
@@ -362,8 +379,8 @@ __device__ __forceinline__ void redecide_band(int gtid, const HeadMeta& hm, cons
 
 // Stages a4 + a3 from the keys alone (any n): MSB radix select over all keys, 11 + 11 + 10 bits,
 // then one pass for the softmax denominator, the bitmap and the threshold band.
-template <class G, bool BY_POS = false>
-__device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+template <class G, bool BY_POS = false, class KeysT>
+__device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta& hm, KeysT keys, uint32_t kmax,
                                                        float kabs, const PostScratch& sc, int r, int S_max,
                                                        const sparq_half* __restrict__ Kt_head, int t_stride = 1) {
     const int lane = gtid & 31, warp = gtid >> 5;
@@ -386,7 +403,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
             zero_hist<G>(sc.hist, gtid);
             G::sync();
             for (int t = gtid; t < n; t += G::NT) {
-                const uint32_t u = keys[t];
+                const uint32_t u = key_full(keys, t);
                 if ((u & mask) == prefix) atomicAdd(&sc.hist[(u >> shift) & ((1u << bits) - 1)], 1u);
             }
             G::sync();
@@ -413,7 +430,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
     float zpart = 0.f;
     for (int wi = warp; wi < nwords; wi += G::NW) {
         const int t = (wi << 5) + lane;
-        const uint32_t u = t < hm.n ? keys[t] : 0u;
+        const uint32_t u = t < hm.n ? key_full(keys, t) : 0u;
         zpart += t < hm.n ? ex2((unkey32(u) - vmax) * c1) : 0.f;
         const bool valid = t < n;
         const bool ge = valid && u >= edge;
@@ -440,7 +457,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
             need_tie = need64;
             for (int wi = warp; wi < nwords; wi += G::NW) {
                 const int t = (wi << 5) + lane;
-                const uint32_t u = t < n ? keys[t] : 0u;
+                const uint32_t u = t < n ? key_full(keys, t) : 0u;
                 const unsigned g = __ballot_sync(FULL, t < n && u > hi_key);
                 const unsigned te = __ballot_sync(FULL, t < n && u >= lo_key && u <= hi_key);
                 if (lane == 0) { sc.bm_sel[wi] = g; sc.bm_tie[wi] = te; }
@@ -456,7 +473,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
                 zero_hist<G>(sc.hist, gtid);
                 G::sync();
                 for (int t = gtid; t < n; t += G::NT) {
-                    const uint32_t u = keys[t];
+                    const uint32_t u = key_full(keys, t);
                     if (u >= lo_key && u <= hi_key) {
                         const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t, t_stride));
                         if ((v & m64) == p64) atomicAdd(&sc.hist[(uint32_t)(v >> shift) & 255u], 1u);
@@ -471,7 +488,7 @@ __device__ __forceinline__ SelectResult select_generic(int gtid, const HeadMeta&
             need_tie = left;
             for (int wi = warp; wi < nwords; wi += G::NW) {
                 const int t = (wi << 5) + lane;
-                const uint32_t u = t < n ? keys[t] : 0u;
+                const uint32_t u = t < n ? key_full(keys, t) : 0u;
                 bool s_ = t < n && u > hi_key, tie = false;
                 if (t < n && u >= lo_key && u <= hi_key) {
                     const unsigned long long v = key64(dot64_at(Kt_head, hm, S_max, r, t, t_stride));
@@ -504,8 +521,8 @@ constexpr int LIST_MAX = HIST_BINS / 2;  // (key, position) pairs of the thresho
 // holds more keys than the list (with WIDE) or a warp's segment of it (without) has room for, or the
 // band reaches outside the bin or holds too many keys -- and the caller runs select_generic instead.
 // Z_stream: the softmax denominator relative to the largest key, accumulated by the stream stage.
-template <class G, int FB_ = FB, bool WIDE = false, bool BY_POS = false>
-__device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+template <class G, int FB_ = FB, bool WIDE = false, bool BY_POS = false, class KeysT>
+__device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, KeysT keys, uint32_t kmax,
                                                  float kabs, float Z_stream, const PostScratch& sc, uint32_t* hist1, int r,
                                                  int S_max, const sparq_half* __restrict__ Kt_head, SelectResult& out,
                                                  int t_stride = 1) {
@@ -578,6 +595,42 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
                 }
             }
         }
+    } else if constexpr (keys_split<KeysT>::value) {
+        // Split keys: the upper halves of eight consecutive keys are one 16-byte vector of shared memory.
+        // A lane owns such a vector -- one load, one whole byte of the bitmap -- and the bin's own keys
+        // go to the one list of the group, as above; their lower halves are fetched after the scan.
+        unsigned char* bm8 = reinterpret_cast<unsigned char*>(sc.bm_sel);
+        uint32_t* list_key = sc.hist;
+        int32_t* list_pos = reinterpret_cast<int32_t*>(sc.hist + LIST_MAX);
+        constexpr int HSH = FSH_ - 16;                       // the first digit inside an upper half
+        for (int v = gtid; v < nwords * 4; v += G::NT) {     // (the bytes of the last word past n are written too, as zeros)
+            const int t = v << 3;
+            const uint4 kv = t < n ? *reinterpret_cast<const uint4*>(keys.hi + t) : make_uint4(0u, 0u, 0u, 0u);
+            const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+            uint32_t sel8 = 0, inb = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const uint32_t dig = ((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xffffu)) >> HSH;
+                sel8 |= (dig > b1) ? 1u << e : 0u;
+                inb |= (dig == b1) ? 1u << e : 0u;
+            }
+            const int rem = n - t;                           // valid positions among the eight
+            if (rem < 8) { const uint32_t vm = rem > 0 ? (1u << rem) - 1u : 0u; sel8 &= vm; inb &= vm; }
+            bm8[v] = (unsigned char)sel8;
+            if (inb) {
+                uint32_t slot = atomicAdd(&sc.band[3], (uint32_t)__popc(inb));
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if ((inb >> e) & 1u) {
+                        if (slot < (uint32_t)LIST_MAX) {
+                            list_key[slot] = ((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xffffu)) << 16;
+                            list_pos[slot] = t + e;
+                        }
+                        ++slot;
+                    }
+                }
+            }
+        }
     } else {
         for (int w0 = warp; w0 < nwords; w0 += 4 * G::NW) {      // four words in flight per warp
             uint32_t u[4];
@@ -586,7 +639,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
             for (int x = 0; x < 4; ++x) {
                 const int t = ((w0 + x * G::NW) << 5) + lane;
                 valid[x] = t < n;                                // also false for words past the end
-                u[x] = valid[x] ? keys[t] : 0u;
+                u[x] = valid[x] ? key_coarse(keys, t) : 0u;
             }
     #pragma unroll
             for (int x = 0; x < 4; ++x) {
@@ -611,9 +664,10 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     out.Z = Z_stream;
     out.need_tie = 0;
     POST_CLK(1);
+    constexpr bool ONE_LIST = WIDE || keys_split<KeysT>::value;   // one list of the group, or a segment per warp
     uint32_t m = 0;
     bool fits = true;
-    if constexpr (WIDE) {
+    if constexpr (ONE_LIST) {
         m = sc.band[3];
         fits = m <= (uint32_t)LIST_MAX;
     } else {
@@ -622,10 +676,14 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     }
     if (!fits) return false;
     // this thread's walk over the list(s): its warp's segment, or its share of the group's one list
-    const uint32_t* my_key = WIDE ? sc.hist : seg_key;
-    const int32_t* my_pos = WIDE ? reinterpret_cast<const int32_t*>(sc.hist + LIST_MAX) : seg_pos;
-    const uint32_t my_first = WIDE ? (uint32_t)gtid : (uint32_t)lane, my_step = WIDE ? (uint32_t)G::NT : 32u;
-    const uint32_t my_n = WIDE ? m : min(wcount, (uint32_t)SEG);
+    uint32_t* my_key = ONE_LIST ? sc.hist : seg_key;
+    const int32_t* my_pos = ONE_LIST ? reinterpret_cast<const int32_t*>(sc.hist + LIST_MAX) : seg_pos;
+    const uint32_t my_first = ONE_LIST ? (uint32_t)gtid : (uint32_t)lane, my_step = ONE_LIST ? (uint32_t)G::NT : 32u;
+    const uint32_t my_n = ONE_LIST ? m : min(wcount, (uint32_t)SEG);
+    if constexpr (keys_split<KeysT>::value) {
+        // the scan listed the keys' upper halves; every thread completes the entries it walks below
+        for (uint32_t i = my_first; i < my_n; i += my_step) my_key[i] |= (uint32_t)__ldcg(keys.lo + my_pos[i]);
+    }
 
     // the threshold among the bin's m keys: `need` of them are wanted; remaining bits as 8 + 8 + the rest
     uint32_t need = (uint32_t)k_eff - above, prefix = b1 << FSH_, mask = ~0u << FSH_, ceq = m;
@@ -633,50 +691,63 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
     // histogram for itself: one barrier per pass instead of three.
     static_assert(CAND_MAX * 12 >= 3 * 256 * 4, "three histograms fit cand_val + cand_pos, free until the band step");
     uint32_t* h256 = reinterpret_cast<uint32_t*>(sc.cand_val);
-    int shift = FSH_;
-    if (ceq != need) {
+    const float twoB = two_b(r, hm.l1_sel, kabs);
+    int shift = FSH_, pass = 0;
+    bool cleared = ceq != need;
+    if (cleared) {
         for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
         G::sync();
     }
+    // Round 0 stops as soon as a whole (sub-)bin is wanted: `prefix` is then that bin's lower edge, not a
+    // key.  If that edge lies so low in the first-digit bin that the 2B band below it would leave the
+    // bin (typically: every key of the bin is wanted, one unit in a few hundred), round 1 goes on to the
+    // exact smallest wanted key, whose band almost surely stays inside.
 #pragma unroll 1
-    for (int pass = 0; pass < 3 && ceq != need; ++pass) {
-        const int bits = pass < 2 ? 8 : FSH_ - 16;
-        shift -= bits;
-        uint32_t* hcur = h256 + pass * 256;
-        for (uint32_t i = my_first; i < my_n; i += my_step) {
-            const uint32_t u = my_key[i];
-            if ((u & mask) == prefix) atomicAdd(&hcur[(u >> shift) & ((1u << bits) - 1)], 1u);
-        }
-        G::sync();
-        // 8 bins per lane, from the top; the lane whose range holds the need-th key knows the answer
-        uint32_t c[8], sum = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { c[i] = hcur[255 - (lane * 8 + i)]; sum += c[i]; }
-        uint32_t incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
-        uint32_t run = incl - sum, bin = 0, cnt = 0;
-        const bool mine = run < need && need <= incl;
-        if (mine) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (run + c[i] >= need) { bin = 255 - (lane * 8 + i); cnt = c[i]; break; }
-                run += c[i];
+    for (int round = 0; round < 2; ++round) {
+#pragma unroll 1
+        for (; pass < 3 && (round == 1 || ceq != need); ++pass) {
+            const int bits = pass < 2 ? 8 : FSH_ - 16;
+            shift -= bits;
+            uint32_t* hcur = h256 + pass * 256;
+            for (uint32_t i = my_first; i < my_n; i += my_step) {
+                const uint32_t u = my_key[i];
+                if ((u & mask) == prefix) atomicAdd(&hcur[(u >> shift) & ((1u << bits) - 1)], 1u);
             }
+            G::sync();
+            // 8 bins per lane, from the top; the lane whose range holds the need-th key knows the answer
+            uint32_t c[8], sum = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) { c[i] = hcur[255 - (lane * 8 + i)]; sum += c[i]; }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += x; }
+            uint32_t run = incl - sum, bin = 0, cnt = 0;
+            const bool mine = run < need && need <= incl;
+            if (mine) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (run + c[i] >= need) { bin = 255 - (lane * 8 + i); cnt = c[i]; break; }
+                    run += c[i];
+                }
+            }
+            const int src = __ffs(__ballot_sync(FULL, mine)) - 1;    // exactly one lane
+            bin = __shfl_sync(FULL, bin, src);
+            run = __shfl_sync(FULL, run, src);
+            cnt = __shfl_sync(FULL, cnt, src);
+            prefix |= bin << shift;
+            mask |= ((1u << bits) - 1) << shift;
+            need -= run;
+            ceq = cnt;
         }
-        const int src = __ffs(__ballot_sync(FULL, mine)) - 1;    // exactly one lane
-        bin = __shfl_sync(FULL, bin, src);
-        run = __shfl_sync(FULL, run, src);
-        cnt = __shfl_sync(FULL, cnt, src);
-        prefix |= bin << shift;
-        mask |= ((1u << bits) - 1) << shift;
-        need -= run;
-        ceq = cnt;
+        if (pass == 3 || (key32(__fadd_rd(unkey32(prefix), -twoB)) >> FSH_) == b1) break;   // (uniform)
+        if (round == 0 && !cleared) {
+            for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
+            G::sync();
+        }
     }
     POST_CLK(2);
     const uint32_t edge = prefix;                            // unprocessed low bits are zero
     const uint32_t over = ceq - need;
-    const float twoB = two_b(r, hm.l1_sel, kabs);
     const float edge_val = unkey32(edge);
     const uint32_t lo_key = key32(__fadd_rd(edge_val, -twoB)), hi_key = key32(__fadd_ru(edge_val, twoB));
     if ((lo_key >> FSH_) != b1 || (hi_key >> FSH_) != b1) return false;   // keys outside the list may be in the band
@@ -703,9 +774,9 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, c
 
 // Local window, before a select that starts from a first-digit histogram of all n keys: take the
 // window's keys out of it again (at most SPARQ_K_MAX of them).  Ends with a barrier.
-template <class G, int FB_ = FB>
-__device__ __forceinline__ void window_unhist(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t* hist1) {
-    for (int t = hm.n_sel + gtid; t < hm.n; t += G::NT) atomicSub(&hist1[keys[t] >> (32 - FB_)], 1u);
+template <class G, int FB_ = FB, class KeysT>
+__device__ __forceinline__ void window_unhist(int gtid, const HeadMeta& hm, KeysT keys, uint32_t* hist1) {
+    for (int t = hm.n_sel + gtid; t < hm.n; t += G::NT) atomicSub(&hist1[key_coarse(keys, t) >> (32 - FB_)], 1u);
     G::sync();
 }
 
@@ -725,13 +796,13 @@ __device__ __forceinline__ void window_mark(int gtid, const HeadMeta& hm, const 
 
 // Local window as large as the budget (k_sel = 0): nothing is ranked.  Clears the bitmap words of the
 // older positions; Z = the softmax denominator relative to the largest key, from the keys.
-template <class G>
-__device__ __forceinline__ SelectResult select_nothing(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax,
+template <class G, class KeysT>
+__device__ __forceinline__ SelectResult select_nothing(int gtid, const HeadMeta& hm, KeysT keys, uint32_t kmax,
                                                        const PostScratch& sc) {
     const float vmax = unkey32(kmax), c1 = hm.inv_tau * LOG2E;
     for (int wi = gtid; wi < ((hm.n_sel + 31) >> 5); wi += G::NT) sc.bm_sel[wi] = 0u;
     float zpart = 0.f;
-    for (int t = gtid; t < hm.n; t += G::NT) zpart += ex2((unkey32(keys[t]) - vmax) * c1);
+    for (int t = gtid; t < hm.n; t += G::NT) zpart += ex2((unkey32(key_full(keys, t)) - vmax) * c1);
     SelectResult res;
     res.Z = group_sum<G>(zpart, sc.red, gtid);               // its barriers publish the bitmap
     res.need_tie = 0;
@@ -778,8 +849,8 @@ __device__ __forceinline__ void build_index_list(int gtid, const HeadMeta& hm, S
 // realloc = false leaves Step 3 out (out = the restricted attention; alpha is still reported).
 // Writes out_row (fp16), alpha_out and idx_k_row when not NULL.  Ends with every thread of the
 // group past its last read of keys and scratch except sc.i2 (read by the idx_k copy at the end).
-template <class G, int RG>
-__device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint32_t* keys, uint32_t kmax, SelectResult sel,
+template <class G, int RG, class KeysT>
+__device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, KeysT keys, uint32_t kmax, SelectResult sel,
                                        const PostScratch& sc, int k, const sparq_half* __restrict__ K_head,
                                        const sparq_half* __restrict__ V_head, const sparq_half* __restrict__ vbar_head,
                                        sparq_half* __restrict__ out_row, int32_t* __restrict__ idx_k_row,
@@ -800,7 +871,7 @@ __device__ __forceinline__ void finish(int gtid, const HeadMeta& hm, const uint3
     }
     // alpha = approximate-score mass of the selected set (Step 3)
     float apart = 0.f;
-    for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(keys[min(max(sc.i2[j], 0), n - 1)]) - vmax) * c1);
+    for (int j = gtid; j < k_eff; j += G::NT) apart += ex2((unkey32(key_full(keys, min(max(sc.i2[j], 0), n - 1))) - vmax) * c1);
     // (numerator and denominator are fp32 sums taken in different orders: keep the mass a probability)
     const float alpha = fminf(group_sum<G>(apart, sc.red, gtid) / Z, 1.0f);
     POST_CLK(4);

@@ -40,11 +40,16 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
 
 // sparq_decode_pipe.cu: persistent warp-specialised variant for S_max small enough that three key
 // buffers, the copy ring and two post-phase scratch areas fit in shared memory
+// Split-key form (the keys' upper halves in shared memory, the lower halves in pipe_split_workspace()
+// bytes of the caller's workspace): reaches caches about three times as long.
 bool pipe_fits(int S_max, int smem_optin);
+bool pipe_split_fits(int S_max, int smem_optin);
+size_t pipe_split_workspace(int S_max, int n_sm);
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream);
+                                     int32_t* status, int n_sm, unsigned int* unit_counter, bool split_keys,
+                                     cudaStream_t stream);
 
 // sparq_decode_wide.cu: one CTA of 512 threads per unit, for a handful of units (batch-1 latency)
 bool wide_fits(int S_max, int smem_optin);

@@ -28,21 +28,28 @@ constexpr int NPROD = 2;                 // producer warps (one warp alone canno
 constexpr int LEAD = 32 * (NPROD + 1);   // producer warps + a1 warp
 constexpr int NT = LEAD + SNT + NPOST * GNT;
 constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
-constexpr int RB = 8;                    // Kt rows per ring stage (32 KB stages: fewer hand-offs beat a deeper ring, measured)
-constexpr int STAGES = 3;
-constexpr int STAGE_BYTES = RB * CH * 2;
-constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+// The ring: RB Kt rows per stage.  32-bit keys: 3 stages of 8 rows (32 KB stages: fewer hand-offs beat a
+// deeper ring, measured).  Split keys (K16: the keys' upper halves in shared memory, the lower halves
+// in the caller's workspace, where the L2 keeps them) are for caches whose 32-bit keys do not fit three
+// times beside that ring: 4 stages of 4 rows, 64 KB.
+template <bool K16>
+struct Ring {
+    static constexpr int RB = K16 ? 4 : 8;
+    static constexpr int STAGES = K16 ? 4 : 3;
+    static constexpr int STAGE_BYTES = RB * CH * 2;
+    static constexpr int BYTES = STAGES * STAGE_BYTES;
+};
+constexpr int STAGES_MAX = 4;
 constexpr int NKB_MAX = 4;               // key buffers: one being written, the others waiting for or in the post groups;
                                          // four where they fit (1.7 us faster on the bench shape), else three
 constexpr int NMETA = 4;                 // unit metadata slots in flight
 using SG = Group<SNT, 1>;
 using PG0 = Group<GNT, 2>;
 using PG1 = Group<GNT, 3>;
-static_assert(RB <= 8, "HeadMeta::qh padding");
 
 // Optional cycle counters for tuning (-DSPARQ_PHASE_CLOCKS): [0] post phase, [1] post waiting for keys,
 // [2] stream waiting for a free key buffer, [3] stream waiting for ring data, [4] stream total per unit,
-// [5] producer waiting for a free ring slot, [6] producer a1
+// [5] producer waiting for a free ring slot, [6] producer a1, [7] units that took the generic select (a count)
 #ifdef SPARQ_PHASE_CLOCKS
 __device__ unsigned long long g_cta_end[256];
 __device__ unsigned long long g_cta_begin[256];
@@ -57,7 +64,7 @@ __device__ unsigned long long g_pipe_clocks[16];
 struct PipeShared {
     HeadMeta meta[NMETA];
     int32_t i2[NPOST][SPARQ_K_MAX];
-    uint64_t full[STAGES], empty[STAGES];          // ring stage landed / consumed
+    uint64_t full[STAGES_MAX], empty[STAGES_MAX];          // ring stage landed / consumed
     uint64_t meta_full[NMETA], meta_free[NMETA];   // a1 done / unit finished
     uint64_t keys_full[NKB_MAX], keys_free[NKB_MAX];   // keys of a unit complete / post-processed
     uint32_t kmax[NKB_MAX];
@@ -72,6 +79,7 @@ struct PipeShared {
     int abort_flag;
 };
 
+constexpr size_t SPLIT_LO_OFFSET = 256;
 struct Args {
     const sparq_half *q, *K, *Kt, *V, *vbar;
     const int32_t* seq_lens;
@@ -80,8 +88,17 @@ struct Args {
     int32_t *idx_r, *idx_k;
     float* alpha;
     int32_t* status;
-    unsigned int* unit_counter;   // zeroed device word for dynamic unit assignment, or NULL: static stride
+    unsigned int* unit_counter;   // zeroed device word for dynamic unit assignment, or NULL: static stride; with split
+                                  // keys their lower halves follow SPLIT_LO_OFFSET bytes behind it, [gridDim.x][NKB][S_cap]
 };
+
+// (A member of its own for this pointer made the struct larger and every instantiation of the kernel
+// spill a few registers, the ones that never use it included.)
+template <int NKB>
+__device__ __forceinline__ uint16_t* split_lo(const Args& a, int kb) {
+    return reinterpret_cast<uint16_t*>(reinterpret_cast<unsigned char*>(a.unit_counter) + SPLIT_LO_OFFSET) +
+           ((size_t)blockIdx.x * NKB + kb) * a.S_cap;
+}
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -124,6 +141,7 @@ __device__ __forceinline__ int next_unit(const Args& a, int bh, int lane) {
     return u < a.n_units ? u : -1;
 }
 
+template <int RB>
 __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uint32_t opts) {
     const int lane = threadIdx.x & 31;
     int bh = (int)blockIdx.x < a.n_units ? (int)blockIdx.x : -1;
@@ -214,7 +232,9 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uin
 }
 
 // ---------------------------------------------------------------------------------- producer
+template <bool K16>
 __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int p) {
+    constexpr int RB = Ring<K16>::RB, STAGES = Ring<K16>::STAGES, STAGE_BYTES = Ring<K16>::STAGE_BYTES;
     const int lane = threadIdx.x & 31;
     const int g_heads = a.Hq / a.Hkv;
     uint32_t g = 0;                                          // ring stages issued so far
@@ -248,16 +268,17 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
 }
 
 // ---------------------------------------------------------------------------------- stream group
-template <int NKB>
+template <int NKB, bool K16>
 __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
                                             uint32_t* hist1_all) {
+    constexpr int RB = Ring<K16>::RB, STAGES = Ring<K16>::STAGES, STAGE_BYTES = Ring<K16>::STAGE_BYTES;
     const int gtid = threadIdx.x - LEAD, lane = gtid & 31;
     int s = 0;                                               // ring slot and its phase parity
     uint32_t parity = 0;
     for (int j = 0, markers = 0; markers < NPOST; ++j) {
         const int m = j % NMETA, kb = j % NKB;
         const HeadMeta& hm = sh.meta[m];
-        uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
+        uint32_t* keys = keys_all + (size_t)kb * a.S_cap / (K16 ? 2 : 1);     // split keys: the upper halves, 2 bytes each
         uint32_t* hist1 = hist1_all + kb * FBINS;
         CLK_BEGIN(t_unit);
 #ifdef SPARQ_PHASE_CLOCKS
@@ -318,14 +339,33 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
                     zm = nm;
                 }
                 if (nvalid >= 8) {
-                    *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
-                    *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
+                    if constexpr (K16) {
+                        uint16_t* keys_hi = reinterpret_cast<uint16_t*>(keys);
+                        uint16_t* keys_lo = split_lo<NKB>(a, kb);
+                        *reinterpret_cast<uint4*>(keys_hi + t0) =
+                            make_uint4(__byte_perm(kk[0], kk[1], 0x7632), __byte_perm(kk[2], kk[3], 0x7632),
+                                       __byte_perm(kk[4], kk[5], 0x7632), __byte_perm(kk[6], kk[7], 0x7632));
+                        __stcg(reinterpret_cast<uint4*>(keys_lo + t0),
+                               make_uint4(__byte_perm(kk[0], kk[1], 0x5410), __byte_perm(kk[2], kk[3], 0x5410),
+                                          __byte_perm(kk[4], kk[5], 0x5410), __byte_perm(kk[6], kk[7], 0x5410)));
+                    } else {
+                        *reinterpret_cast<uint4*>(keys + t0) = make_uint4(kk[0], kk[1], kk[2], kk[3]);
+                        *reinterpret_cast<uint4*>(keys + t0 + 4) = make_uint4(kk[4], kk[5], kk[6], kk[7]);
+                    }
 #pragma unroll
                     for (int e = 0; e < 8; ++e) { kmax = max(kmax, kk[e]); atomicAdd(&hist1[kk[e] >> FSH], 1u); }
                 } else {
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
-                        if (e < nvalid) { keys[t0 + e] = kk[e]; kmax = max(kmax, kk[e]); atomicAdd(&hist1[kk[e] >> FSH], 1u); }
+                        if (e < nvalid) {
+                            if constexpr (K16) {
+                                reinterpret_cast<uint16_t*>(keys)[t0 + e] = (uint16_t)(kk[e] >> 16);
+                                __stcg(split_lo<NKB>(a, kb) + t0 + e, (uint16_t)(kk[e] & 0xffffu));
+                            }
+                            else keys[t0 + e] = kk[e];
+                            kmax = max(kmax, kk[e]);
+                            atomicAdd(&hist1[kk[e] >> FSH], 1u);
+                        }
                 }
             }
             uint32_t kabs_bits = __float_as_uint(mx_to_float(mx));
@@ -344,7 +384,7 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 }
 
 // ---------------------------------------------------------------------------------- post groups
-template <class PG, int NKB>
+template <class PG, int NKB, bool K16>
 __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, uint32_t* hist1_all,
                                           unsigned char* scratch, int p, const uint32_t opts) {
     const int gtid = threadIdx.x - LEAD - SNT - p * GNT;
@@ -376,8 +416,15 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             if (gtid < D) out_row[gtid] = a.vbar[kv_head * D + gtid];
             if (gtid == 0 && a.alpha) a.alpha[bh] = 0.f;
         } else {
-            const uint32_t* keys = keys_all + (size_t)kb * a.S_cap;
             const sparq_half* Kt_head = a.Kt + kv_head * (size_t)D * a.S_max;
+            auto keys = [&] {
+                if constexpr (K16) {
+                    return SplitKeys{reinterpret_cast<const uint16_t*>(keys_all) + (size_t)kb * a.S_cap,
+                                     split_lo<NKB>(a, kb)};
+                } else {
+                    return keys_all + (size_t)kb * a.S_cap;
+                }
+            }();
             SelectResult sel;
             const bool windowed = (opts >> 16) != 0u && hm.n_sel != hm.n;   // (uniform) a local window is reserved inside the budget
             if (windowed && hm.k_sel == 0) {                 // the window takes the whole budget: nothing to rank
@@ -386,8 +433,12 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
             } else {
                 if (windowed) window_unhist<PG>(gtid, hm, keys, hist1_all + kb * FBINS);
                 if (!select_prefilled<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sh.zsum[kb], sc, hist1_all + kb * FBINS, a.r,
-                                          a.S_max, Kt_head, sel))
+                                          a.S_max, Kt_head, sel)) {
+#ifdef SPARQ_PHASE_CLOCKS
+                    if (gtid == 0) atomicAdd(&g_pipe_clocks[7], 1ull);
+#endif
                     sel = select_generic<PG>(gtid, hm, keys, sh.kmax[kb], sh.kabs[kb], sc, a.r, a.S_max, Kt_head);
+                }
             }
             if (windowed) window_mark<PG>(gtid, hm, sc);
             finish<PG, 4>(gtid, hm, keys, sh.kmax[kb], sel, sc, a.k, a.K + kv_head * (size_t)a.S_max * D,
@@ -403,19 +454,20 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
 
 // OPT = false: the paper's algorithm as stated, the settings word known to be 0 at compile time (the
 // instantiation the plain decode call runs); OPT = true: settings taken from `opts_arg`.
-template <int NKB, bool OPT>
+template <int NKB, bool OPT, bool K16>
 __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, const uint32_t opts_arg) {
+    using R = Ring<K16>;
     const uint32_t opts = OPT ? opts_arg : 0u;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
-    uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + RING_BYTES);
-    uint32_t* hist1_all = keys_all + (size_t)NKB * a.S_cap;               // per key buffer: histogram of the keys' top bits
+    uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + R::BYTES);     // NKB buffers of S_cap keys (split keys: their upper halves)
+    uint32_t* hist1_all = keys_all + (size_t)NKB * a.S_cap / (K16 ? 2 : 1);   // per key buffer: histogram of the keys' top bits
     unsigned char* scratch0 = reinterpret_cast<unsigned char*>(hist1_all + NKB * FBINS);
     const size_t scratch_bytes = (post_scratch_bytes(GNT / 16, a.S_cap / 32) + 127) & ~(size_t)127;
     __shared__ PipeShared sh;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], SNT / 32); }
+        for (int s = 0; s < R::STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], SNT / 32); }
         for (int m = 0; m < NMETA; ++m) { mbar_init(&sh.meta_full[m], 1); mbar_init(&sh.meta_free[m], 1); }
         for (int b = 0; b < NKB; ++b) { mbar_init(&sh.keys_full[b], 1); mbar_init(&sh.keys_free[b], 1); }
         sh.abort_flag = 0;
@@ -427,17 +479,19 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, 
     if (threadIdx.x == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_cta_begin[blockIdx.x] = gt; g_cta_end[blockIdx.x] = 0; }
 #endif
     const int warp = threadIdx.x >> 5;
-    if (warp < NPROD) producer_role(a, sh, ring, warp);
-    else if (warp == NPROD) a1_role(a, sh, opts);
-    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB>(a, sh, ring, keys_all, hist1_all);
-    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB>(a, sh, keys_all, hist1_all, scratch0, 0, opts);
-    else post_role<PG1, NKB>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1, opts);
+    if (warp < NPROD) producer_role<K16>(a, sh, ring, warp);
+    else if (warp == NPROD) a1_role<R::RB>(a, sh, opts);
+    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB, K16>(a, sh, ring, keys_all, hist1_all);
+    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB, K16>(a, sh, keys_all, hist1_all, scratch0, 0, opts);
+    else post_role<PG1, NKB, K16>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1, opts);
 }
 
-size_t pipe_dynamic_smem(int S_cap, int NKB) {
+size_t pipe_dynamic_smem(int S_cap, int NKB, bool k16) {
     const size_t scratch = (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127;
-    return (size_t)RING_BYTES + (size_t)NKB * S_cap * 4 + (size_t)NKB * FBINS * 4 + NPOST * scratch;
+    return (size_t)(k16 ? Ring<true>::BYTES : Ring<false>::BYTES) + (size_t)NKB * S_cap * (k16 ? 2 : 4) +
+           (size_t)NKB * FBINS * 4 + NPOST * scratch;
 }
+constexpr int NKB_SPLIT = 3;             // key buffers of the split-key form
 
 }  // namespace
 
@@ -465,24 +519,31 @@ extern "C" int sparq_debug_post_clocks(unsigned long long* out16, int reset) {
 // S_max rounded up so that bitmap words and 16-byte key vectors stay whole
 static int pipe_s_cap(int S_max) { return (S_max + 127) & ~127; }
 
-static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb) {
-    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
+static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb, bool k16) {
+    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb, k16) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
 }
-bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3); }
+bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3, false); }
+bool pipe_split_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true); }
+// Workspace of the split-key form: the unit counter, then the keys' lower halves.
+size_t pipe_split_workspace(int S_max, int n_sm) { return SPLIT_LO_OFFSET + (size_t)n_sm * NKB_SPLIT * pipe_s_cap(S_max) * 2; }
 
+// split_keys: unit_counter heads a workspace of pipe_split_workspace() bytes; else 32-bit keys in shared memory.
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
                                      int r, int k, uint32_t opts, sparq_half* out, int32_t* idx_r, int32_t* idx_k, float* alpha,
-                                     int32_t* status, int n_sm, unsigned int* unit_counter, cudaStream_t stream) {
+                                     int32_t* status, int n_sm, unsigned int* unit_counter, bool split_keys,
+                                     cudaStream_t stream) {
     Args a;
     a.q = q; a.K = K; a.Kt = Kt; a.V = V; a.vbar = vbar; a.seq_lens = seq_lens;
     a.n_units = B * Hq; a.Hq = Hq; a.Hkv = Hkv; a.S_max = S_max; a.S_cap = pipe_s_cap(S_max); a.r = r; a.k = k;
     a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status; a.unit_counter = unit_counter;
     const int smem_optin = device_info().smem_optin;
-    const bool four = pipe_fits_nkb(S_max, smem_optin, 4);
-    const size_t dyn = pipe_dynamic_smem(a.S_cap, four ? 4 : 3);
-    auto kernel = opts ? (four ? sparq_decode_pipe_kernel<4, true> : sparq_decode_pipe_kernel<3, true>)
-                       : (four ? sparq_decode_pipe_kernel<4, false> : sparq_decode_pipe_kernel<3, false>);
+    const bool k16 = split_keys && unit_counter;
+    const bool four = !k16 && pipe_fits_nkb(S_max, smem_optin, 4, false);
+    const size_t dyn = pipe_dynamic_smem(a.S_cap, k16 ? NKB_SPLIT : (four ? 4 : 3), k16);
+    auto kernel = k16 ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true>)
+                : opts ? (four ? sparq_decode_pipe_kernel<4, true, false> : sparq_decode_pipe_kernel<3, true, false>)
+                       : (four ? sparq_decode_pipe_kernel<4, false, false> : sparq_decode_pipe_kernel<3, false, false>);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     const int grid = a.n_units < n_sm ? a.n_units : n_sm;

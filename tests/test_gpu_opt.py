@@ -89,7 +89,7 @@ SETTINGS = [
 ]
 
 
-@pytest.mark.parametrize("plan", [None, "simple", "pipe", "split", "wide"])
+@pytest.mark.parametrize("plan", [None, "simple", "pipe", "split", "wide", "pipe16"])
 def test_settings_on_ragged_batch(plan):
     rng = np.random.default_rng(77)
     B, Hq, Hkv, S, r, k = 4, 8, 4, 2304, 32, 128
@@ -206,7 +206,7 @@ def test_random_settings(seed):
     cache = H.DeviceCache(K, V, seq)
     what = "seed %d B=%d Hq=%d Hkv=%d S=%d n=%s r=%d k=%d tau=%d realloc=%d window=%d" % (
         seed, B, Hkv * g, Hkv, S, lens.tolist(), r, k, tau_mode, realloc, window)
-    plans = [None, "simple", "wide", "pipe"]
+    plans = [None, "simple", "wide", "pipe", "pipe16"]
     if sparq.sparq_workspace_bytes(B, Hkv * g, Hkv, 128, S, r, k) == 0 and S >= 2048:
         plans.append("split")
     for plan in plans:

@@ -38,14 +38,14 @@ def test_c0_tiny_single_step_against_numpy_oracle():
     _dense_check(c, cache, c.q_steps[0], "c0")
 
 
-@pytest.mark.parametrize("plan", ["split", "pipe", "simple", "wide"])
+@pytest.mark.parametrize("plan", ["split", "pipe", "simple", "wide", "pipe16"])
 def test_c1_llama2_batch1_all_heads(plan):
     """Batch 1, 32 heads: fewer units than SMs.  The library's own choice at this length is the
     wide kernel (one 512-thread CTA per unit); the sliced plan, the persistent kernel and the
     one-CTA-per-unit kernel must give the same parity."""
     c = synth.make_case("c1")
     with H.decode_plan(plan):
-        assert (sparq.sparq_workspace_bytes(1, 32, 32, 128, 4096, 32, 128) > 0) == (plan == "split")
+        assert (sparq.sparq_workspace_bytes(1, 32, 32, 128, 4096, 32, 128) > 0) == (plan in ("split", "pipe16"))
         waived, total = H.run_case_all_heads(c, "c1 " + plan)
     assert total == 32 and waived <= 1
 
@@ -108,6 +108,19 @@ def test_persistent_kernel_with_three_key_buffers():
     with H.decode_plan("pipe"):
         waived, total = H.run_case_all_heads(c, "three key buffers")
     assert total == 320 and waived <= 2
+
+
+def test_persistent_kernel_with_split_keys():
+    """The persistent kernel's form for caches whose 32-bit keys do not fit its shared memory three
+    times: the keys' upper halves stay in shared memory, the lower halves go through the workspace.
+    More units than SMs on a long ragged GQA cache, so ring, key-buffer and workspace slots wrap."""
+    c = synth.make_case("c3", device="cuda", B=6, S=16384, ragged=(12000, 16383))      # 192 units
+    c.K, c.V, c.q_steps, c.k_steps, c.v_steps, c.seq_lens = (t.cpu() for t in (c.K, c.V, c.q_steps, c.k_steps,
+                                                                                  c.v_steps, c.seq_lens))
+    with H.decode_plan("pipe16"):
+        assert sparq.sparq_workspace_bytes(6, 32, 8, 128, 16384, c.r, c.k) > 0
+        waived, total = H.run_case_all_heads(c, "split keys")
+    assert total == 192 and waived <= 2
 
 
 def test_split_plan_unsliced_many_units():

@@ -59,7 +59,7 @@ def test_random_shape(seed):
     ora = c_oracle.sparq_decode(qn, Knp, Vnp, seq.numpy(), r, k)
     units = (qn.reshape(B * Hq, -1), lambda u: Knp[u // Hq, (u % Hq) // g], lambda u: Vnp[u // Hq, (u % Hq) // g],
              np.repeat(seq.numpy(), Hq))
-    plans = [None, "simple", "wide"] + (["pipe"] if S <= 5000 else [])
+    plans = [None, "simple", "wide"] + (["pipe"] if S <= 5000 else []) + (["pipe16"] if S <= 17000 else [])
     if sparq.sparq_workspace_bytes(B, Hq, Hkv, 128, S, r, k) == 0 and S >= 2048:
         plans.append("split")                                 # (forced; short caches have no split plan)
     for plan in plans:
