@@ -35,16 +35,17 @@ PERIOD = 64          # steps between rewinds of seq_lens (the cache would otherw
 POOL = 16            # distinct (q, k_new, v_new) sets rotated through the steps
 L2_BYTES = 126e6
 EV_EVERY = 4          # steps between CUDA-event pairs around the decode inside the timed region
-# which decode kernel the library picks per workload (caches too long for the persistent kernel's
-# shared memory take the wide kernel); every step launches the append kernel and one decode kernel
-DECODE_KERNEL = {"c1": "sparq_decode_wide_kernel", "c3": "sparq_decode_wide_kernel", "c4": "sparq_decode_wide_kernel"}
+# which decode kernel the library picks per workload (the persistent kernel on c2 and, in its split-key
+# form, on c3; the wide kernel for one unit per SM and for c4's long cache); every step launches the
+# append kernel and one decode kernel
+DECODE_KERNEL = {"c1": "sparq_decode_wide_kernel", "c4": "sparq_decode_wide_kernel"}
 LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one sparq_decode_kernel launch on this workload,
 # from the ncu capture summarised under profiles/ (None until a capture exists).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     "c2": 681.0e6,   # 2 x (336.47 + 4.05) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md (B = 32 capture, scaled by the units)
-    "c3": 508.5e6,   # 505.1 + 3.4 MB: profiles/sparq_decode_wide_kernel_c3_c4.md
+    "c3": 540.9e6,   # 510.4 + 30.5 MB: profiles/sparq_decode_pipe_kernel_split_keys_c3.md (the keys' lower halves are written out)
     "c4": 812.5e6,   # 808.8 + 3.7 MB: the same file (the heads of a group share rows in the L2)
 }
 

@@ -156,6 +156,19 @@ static bool split_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok)
 // CTA per SM: 260 against 289).
 static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= n_sm || !pipe_ok; }
 
+// The persistent kernel's split-key form against the wide kernel, for caches too long for the persistent
+// kernel's 32-bit keys: with four or more units per SM its hand-built overlap of one unit's stream with
+// the others' select and gather beats the wide kernel's two CTAs per SM (1024 units of 16384 positions
+// at r = 16: 122 against 142 us; 2048 units of 8192 at r = 16: 125 against 156; 1024 units of 8192 at
+// r = 32: 117 against 132), with fewer it loses (256 units of 16384: 48 against 41).  Beyond about 11,800
+// positions only a 64 KB ring fits beside the keys, which holds the stream back when the rows are many
+// (1024 units of 16384 at r = 32: 201 against 195; 512 units at r = 64: 223 against 175): there only up to r = 16.
+static bool pipe16_preferred(int units, int S_max, int r, int n_sm) {
+    const int smem = device_info().smem_optin;
+    if (units < 4 * n_sm || pipe_fits(S_max, smem) || !pipe_split_fits(S_max, smem)) return false;
+    return !pipe_split_thin_ring(S_max, smem) || r <= 16;
+}
+
 // Two 256-thread CTAs per SM instead of one of 512 threads: with more units than SMs, where both fit.
 // SPARQ_WIDE_PAIRS=0|1 overrides (tuning).
 static bool wide_pairs(int units, int S_max, int n_sm) {
@@ -174,6 +187,7 @@ size_t sparq_workspace_bytes(int B, int Hq, int Hkv, int d, int S_max, int r, in
     const bool pipe_ok = pipe_fits(S_max, device_smem_optin());
     const int plan = forced_plan();                          // a plan forced through the environment gets what it needs
     if (plan == 5) return pipe_split_fits(S_max, device_smem_optin()) ? pipe_split_bytes(S_max, n_sm) : 0;
+    if (plan == 0 && pipe16_preferred(B * Hq, S_max, r, n_sm)) return pipe_split_bytes(S_max, n_sm);
     if (plan == 4 || (plan == 0 && wide_fits(S_max, device_smem_optin()) && wide_preferred(B * Hq, n_sm, pipe_ok)))
         return 0;
     if (splits && (plan == 3 || (plan == 0 && split_preferred(B * Hq, S_max, r, n_sm, pipe_ok))))
@@ -202,9 +216,11 @@ static int decode_with(const sparq_half* q, const sparq_half* K, const sparq_hal
     if (plan == 3 && !ws_ok) return SPARQ_ERR_WORKSPACE;
     // one 512-thread CTA per unit with the keys in shared memory: the choice for a handful of units whatever
     // their length, and beside the split plan for caches the persistent kernel cannot hold
-    if (plan == 5) {
+    // the persistent kernel's split-key form: the library's choice only with its workspace (without, the wide kernel)
+    const bool p16_ws = workspace && workspace_bytes >= pipe_split_bytes(S_max, n_sm);
+    if (plan == 5 || (plan == 0 && p16_ws && pipe16_preferred(B * Hq, S_max, r, n_sm))) {
         if (!pipe_split_fits(S_max, device_smem_optin())) return SPARQ_ERR_TOO_LONG;
-        if (!workspace || workspace_bytes < pipe_split_bytes(S_max, n_sm)) return SPARQ_ERR_WORKSPACE;
+        if (!p16_ws) return SPARQ_ERR_WORKSPACE;
         return rc(launch_sparq_decode_pipe(q, K, Kt, V, vbar, seq_lens, B, Hq, Hkv, S_max, r, k, opts, out, idx_r, idx_k,
                                            alpha, status, n_sm, static_cast<unsigned int*>(workspace), true,
                                            (cudaStream_t)stream));

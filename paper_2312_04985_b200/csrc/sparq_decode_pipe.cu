@@ -28,14 +28,14 @@ constexpr int NPROD = 2;                 // producer warps (one warp alone canno
 constexpr int LEAD = 32 * (NPROD + 1);   // producer warps + a1 warp
 constexpr int NT = LEAD + SNT + NPOST * GNT;
 constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream thread (one 16-byte vector)
-// The ring: RB Kt rows per stage.  32-bit keys: 3 stages of 8 rows (32 KB stages: fewer hand-offs beat a
-// deeper ring, measured).  Split keys (K16: the keys' upper halves in shared memory, the lower halves
-// in the caller's workspace, where the L2 keeps them) are for caches whose 32-bit keys do not fit three
-// times beside that ring: 4 stages of 4 rows, 64 KB.
-template <bool K16>
+// The ring: RB Kt rows per stage.  3 stages of 8 rows (32 KB stages: fewer hand-offs beat a deeper ring,
+// measured), or, where the longest caches of the split-key form leave less room, 4 stages of 4 rows (64 KB).
+// Split keys (K16): the keys' upper halves in shared memory, the lower halves in the caller's workspace,
+// where the L2 keeps them; for caches whose 32-bit keys do not fit three times beside the ring.
+template <bool THIN>
 struct Ring {
-    static constexpr int RB = K16 ? 4 : 8;
-    static constexpr int STAGES = K16 ? 4 : 3;
+    static constexpr int RB = THIN ? 4 : 8;
+    static constexpr int STAGES = THIN ? 4 : 3;
     static constexpr int STAGE_BYTES = RB * CH * 2;
     static constexpr int BYTES = STAGES * STAGE_BYTES;
 };
@@ -232,9 +232,9 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uin
 }
 
 // ---------------------------------------------------------------------------------- producer
-template <bool K16>
+template <bool THIN>
 __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int p) {
-    constexpr int RB = Ring<K16>::RB, STAGES = Ring<K16>::STAGES, STAGE_BYTES = Ring<K16>::STAGE_BYTES;
+    constexpr int RB = Ring<THIN>::RB, STAGES = Ring<THIN>::STAGES, STAGE_BYTES = Ring<THIN>::STAGE_BYTES;
     const int lane = threadIdx.x & 31;
     const int g_heads = a.Hq / a.Hkv;
     uint32_t g = 0;                                          // ring stages issued so far
@@ -268,10 +268,10 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
 }
 
 // ---------------------------------------------------------------------------------- stream group
-template <int NKB, bool K16>
+template <int NKB, bool K16, bool THIN>
 __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
                                             uint32_t* hist1_all) {
-    constexpr int RB = Ring<K16>::RB, STAGES = Ring<K16>::STAGES, STAGE_BYTES = Ring<K16>::STAGE_BYTES;
+    constexpr int RB = Ring<THIN>::RB, STAGES = Ring<THIN>::STAGES, STAGE_BYTES = Ring<THIN>::STAGE_BYTES;
     const int gtid = threadIdx.x - LEAD, lane = gtid & 31;
     int s = 0;                                               // ring slot and its phase parity
     uint32_t parity = 0;
@@ -454,9 +454,9 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
 
 // OPT = false: the paper's algorithm as stated, the settings word known to be 0 at compile time (the
 // instantiation the plain decode call runs); OPT = true: settings taken from `opts_arg`.
-template <int NKB, bool OPT, bool K16>
+template <int NKB, bool OPT, bool K16, bool THIN>
 __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, const uint32_t opts_arg) {
-    using R = Ring<K16>;
+    using R = Ring<THIN>;
     const uint32_t opts = OPT ? opts_arg : 0u;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
@@ -479,16 +479,16 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, 
     if (threadIdx.x == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_cta_begin[blockIdx.x] = gt; g_cta_end[blockIdx.x] = 0; }
 #endif
     const int warp = threadIdx.x >> 5;
-    if (warp < NPROD) producer_role<K16>(a, sh, ring, warp);
+    if (warp < NPROD) producer_role<THIN>(a, sh, ring, warp);
     else if (warp == NPROD) a1_role<R::RB>(a, sh, opts);
-    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB, K16>(a, sh, ring, keys_all, hist1_all);
+    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB, K16, THIN>(a, sh, ring, keys_all, hist1_all);
     else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB, K16>(a, sh, keys_all, hist1_all, scratch0, 0, opts);
     else post_role<PG1, NKB, K16>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1, opts);
 }
 
-size_t pipe_dynamic_smem(int S_cap, int NKB, bool k16) {
+size_t pipe_dynamic_smem(int S_cap, int NKB, bool k16, bool thin) {
     const size_t scratch = (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127;
-    return (size_t)(k16 ? Ring<true>::BYTES : Ring<false>::BYTES) + (size_t)NKB * S_cap * (k16 ? 2 : 4) +
+    return (size_t)(thin ? Ring<true>::BYTES : Ring<false>::BYTES) + (size_t)NKB * S_cap * (k16 ? 2 : 4) +
            (size_t)NKB * FBINS * 4 + NPOST * scratch;
 }
 constexpr int NKB_SPLIT = 3;             // key buffers of the split-key form
@@ -519,11 +519,12 @@ extern "C" int sparq_debug_post_clocks(unsigned long long* out16, int reset) {
 // S_max rounded up so that bitmap words and 16-byte key vectors stay whole
 static int pipe_s_cap(int S_max) { return (S_max + 127) & ~127; }
 
-static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb, bool k16) {
-    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb, k16) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
+static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb, bool k16, bool thin) {
+    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb, k16, thin) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
 }
-bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3, false); }
-bool pipe_split_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true); }
+bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3, false, false); }
+bool pipe_split_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, true); }
+bool pipe_split_thin_ring(int S_max, int smem_optin) { return !pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, false); }
 // Workspace of the split-key form: the unit counter, then the keys' lower halves.
 size_t pipe_split_workspace(int S_max, int n_sm) { return SPLIT_LO_OFFSET + (size_t)n_sm * NKB_SPLIT * pipe_s_cap(S_max) * 2; }
 
@@ -539,11 +540,13 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
     a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status; a.unit_counter = unit_counter;
     const int smem_optin = device_info().smem_optin;
     const bool k16 = split_keys && unit_counter;
-    const bool four = !k16 && pipe_fits_nkb(S_max, smem_optin, 4, false);
-    const size_t dyn = pipe_dynamic_smem(a.S_cap, k16 ? NKB_SPLIT : (four ? 4 : 3), k16);
-    auto kernel = k16 ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true>)
-                : opts ? (four ? sparq_decode_pipe_kernel<4, true, false> : sparq_decode_pipe_kernel<3, true, false>)
-                       : (four ? sparq_decode_pipe_kernel<4, false, false> : sparq_decode_pipe_kernel<3, false, false>);
+    const bool four = !k16 && pipe_fits_nkb(S_max, smem_optin, 4, false, false);
+    const bool thin = k16 && pipe_split_thin_ring(S_max, smem_optin);
+    const size_t dyn = pipe_dynamic_smem(a.S_cap, k16 ? NKB_SPLIT : (four ? 4 : 3), k16, thin);
+    auto kernel = k16 ? (thin ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, true> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, true>)
+                              : (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, false> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, false>))
+                : opts ? (four ? sparq_decode_pipe_kernel<4, true, false, false> : sparq_decode_pipe_kernel<3, true, false, false>)
+                       : (four ? sparq_decode_pipe_kernel<4, false, false, false> : sparq_decode_pipe_kernel<3, false, false, false>);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     const int grid = a.n_units < n_sm ? a.n_units : n_sm;
