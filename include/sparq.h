@@ -127,15 +127,17 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
  * int32 = i2 ascending, unused tail -1; alpha [B,Hq] fp32.
  * workspace: optional device scratch; sparq_workspace_bytes() says how much helps for the given
  * shapes (0: none -- a handful of units, or few units per SM on a long cache, run on a kernel
- * that keeps a unit's approximate scores in shared memory).  Two uses, the selected sets
+ * that keeps a unit's approximate scores in shared memory).  Three uses, the selected sets
  * identical in all plans (alpha and out may differ in their last bits, the softmax denominator
- * being summed in another order): many units on a cache too long for the persistent kernel's
- * shared memory, or any cache beyond sparq_max_seq_len() -- the approximate scores of a unit
- * pass through the workspace (4 bytes per position), and with few units every sequence is cut
- * into slices handled by different thread blocks; more units than SMs on the persistent kernel
- * -- 64 bytes for a counter from which the thread blocks draw their units, which evens out
- * their finishing times.  With workspace NULL or too small a plan without scratch is used.  The
- * call clears what it needs; contents are undefined afterwards.
+ * being summed in another order): a cache beyond sparq_max_seq_len() -- the approximate scores
+ * of a unit pass through the workspace (4 bytes per position), and with few units every sequence
+ * is cut into slices handled by different thread blocks; more units than SMs on the persistent
+ * kernel -- 64 bytes for a counter from which the thread blocks draw their units, which evens
+ * out their finishing times; four or more units per SM on a cache of about 6,000 to 17,000
+ * positions -- the persistent kernel keeps only the upper halves of the scores' sort keys in
+ * shared memory and parks the lower halves here (SMs x 3 x 2 bytes per position).  With
+ * workspace NULL or too small a plan without scratch is used.  The call clears what it needs;
+ * contents are undefined afterwards.
  */
 int sparq_decode(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                  const sparq_half* vbar, const int32_t* seq_lens,
