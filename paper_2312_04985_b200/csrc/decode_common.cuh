@@ -698,14 +698,14 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, K
         for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
         G::sync();
     }
-    // Round 0 stops as soon as a whole (sub-)bin is wanted: `prefix` is then that bin's lower edge, not a
+    // The first go stops as soon as a whole (sub-)bin is wanted: `prefix` is then that bin's lower edge, not a
     // key.  If that edge lies so low in the first-digit bin that the 2B band below it would leave the
-    // bin (typically: every key of the bin is wanted, one unit in a few hundred), round 1 goes on to the
+    // bin (typically: every key of the bin is wanted, one unit in a few hundred), a second go carries on to the
     // exact smallest wanted key, whose band almost surely stays inside.
 #pragma unroll 1
-    for (int round = 0; round < 2; ++round) {
+    for (int go = 0; go < 2; ++go) {
 #pragma unroll 1
-        for (; pass < 3 && (round == 1 || ceq != need); ++pass) {
+        for (; pass < 3 && (go == 1 || ceq != need); ++pass) {
             const int bits = pass < 2 ? 8 : FSH_ - 16;
             shift -= bits;
             uint32_t* hcur = h256 + pass * 256;
@@ -740,7 +740,7 @@ __device__ __forceinline__ bool select_prefilled(int gtid, const HeadMeta& hm, K
             ceq = cnt;
         }
         if (pass == 3 || (key32(__fadd_rd(unkey32(prefix), -twoB)) >> FSH_) == b1) break;   // (uniform)
-        if (round == 0 && !cleared) {
+        if (go == 0 && !cleared) {
             for (int i = gtid; i < 3 * 256; i += G::NT) h256[i] = 0;
             G::sync();
         }
