@@ -43,10 +43,11 @@ bool bad_common(int B, int Hq, int Hkv, int d, int S_max) {
 
 int device_sm_count() { return device_info().sm_count; }
 
-// SPARQ_DECODE_PLAN=simple|pipe|split|wide forces one of the sparq_decode plans (tests and tuning).
+// SPARQ_DECODE_PLAN=simple|pipe|pipe16|split|wide forces one of the sparq_decode plans (tests and tuning).
 // Unset or anything else: the wide kernel (one CTA of 512 threads, or two of 256, per SM; a unit's
-// keys in shared memory) for up to one unit per SM and for caches too long for the persistent
-// kernel; the persistent pipelined kernel wherever else one unit's keys fit its shared memory;
+// keys in shared memory) for up to two units per SM and for caches too long for the persistent
+// kernel; the persistent pipelined kernel wherever else one unit's keys fit its shared memory, and in
+// its split-key form (pipe16) for four or more units per SM on caches up to about 17,000 positions;
 // beyond the wide kernel's reach (about 44,000 positions) the split plan if the caller passed its
 // workspace; else one CTA per unit.
 int forced_plan() {
@@ -154,7 +155,10 @@ static bool split_preferred(int units, int S_max, int r, int n_sm, bool pipe_ok)
 // kernel wins on the longer caches (1024 units of 16384, r = 16, two CTAs per SM: 141 against the
 // split plan's 147 us; 256 units: 43 against 71; 512 units of up to 32800 positions at r = 64, one
 // CTA per SM: 260 against 289).
-static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= n_sm || !pipe_ok; }
+// Up to two units per SM all of them are resident at once as two CTAs per SM, and the wide kernel still
+// wins (4096 positions, r = 32: 160 units 25.3 against the persistent kernel's 28.6 us, 256 units 29.1
+// against 32.2; 320 units 40.2 against 37.9, 1024 units 86.9 against 73.2).
+static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= 2 * n_sm || !pipe_ok; }
 
 // The persistent kernel's split-key form against the wide kernel, for caches too long for the persistent
 // kernel's 32-bit keys: with four or more units per SM its hand-built overlap of one unit's stream with

@@ -21,7 +21,7 @@ ALPHA_TOL = 5e-5    # fp32 exponentials of fp32-rounded logits against the float
 
 @contextlib.contextmanager
 def decode_plan(name):
-    """Force one of the sparq_decode plans ('simple', 'pipe', 'split') or None for the library's choice."""
+    """Force one of the sparq_decode plans ('simple', 'pipe', 'pipe16', 'split', 'wide') or None for the library's choice."""
     old = os.environ.get("SPARQ_DECODE_PLAN")
     if name is None:
         os.environ.pop("SPARQ_DECODE_PLAN", None)
