@@ -267,6 +267,34 @@ def test_fp32_ties_are_decided_in_fp64():
     assert len(set(lh.float().tolist())) == 3 and len(set(lh.tolist())) > 20   # the case is what it claims
 
 
+@pytest.mark.parametrize("plan", [None, "simple", "pipe", "wide", "pipe16"])
+def test_whole_threshold_bin_wanted(plan):
+    """Exactly k scores lie in one half-octave [1, 1.5) and every other score far below: the select's
+    first-digit bin at the threshold holds exactly the wanted keys, its lower edge is the bin's own, and
+    the rounding-error band below that edge reaches into the next bin -- the case in which the short-cut
+    select goes on to the exact smallest wanted key.  Also with k - 3 and k + 5, where the threshold lies
+    inside the bin and inside the next populated one."""
+    rng = np.random.default_rng(21)
+    B, Hq, Hkv, S, r, k = 2, 2, 2, 2048, 1, 64
+    q = torch.from_numpy(rng.standard_normal((B, Hq, 128)) * 0.01).half()
+    q[..., 7] = 4.0                                           # r = 1 keeps component 7
+    K = torch.from_numpy(rng.standard_normal((B, Hkv, S, 128))).half()
+    V = torch.from_numpy(rng.standard_normal((B, Hkv, S, 128))).half()
+    seq = torch.tensor([S, 1500], dtype=torch.int32)
+    for b in range(B):
+        for h in range(Hkv):
+            n = int(seq[b])
+            col = torch.from_numpy(rng.uniform(0.25, 0.5, S)).half()
+            top = rng.choice(n, size=k, replace=False)
+            col[top] = torch.from_numpy(rng.uniform(1.0, 1.499, k)).half()
+            K[b, h, :, 7] = col
+    with H.decode_plan(plan):
+        for kk in (k, k - 3, k + 5):
+            cache, gpu, ora, waived = _compare_all(q, K, V, seq, r, kk, "whole bin plan=%s k=%d" % (plan, kk))
+            assert np.array_equal(gpu["i2"], ora["i2"])
+    assert (gpu["i1"] == 7).all()
+
+
 def test_repeat_launches_are_bitwise_identical():
     c = synth.make_case("c1", Hq=8, Hkv=8)
     cache = H.DeviceCache(c.K, c.V, c.seq_lens + 1)
