@@ -11,7 +11,8 @@ from tests import harness as H
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,kw", [("c1", {}), ("c2", dict(B=6, S=1024)), ("c3", dict(B=1, S=8192))])
+@pytest.mark.parametrize("name,kw", [("c1", {}), ("c2", dict(B=6, S=1024)), ("c3", dict(B=1, S=8192)),
+                                     ("c3", dict(B=19, S=6144))])     # (the last: the persistent kernel with split keys)
 def test_replayed_steps_equal_eager_steps(name, kw):
     n_steps = 3
     c = synth.make_case(name, backend="numpy", n_steps=n_steps, **kw)
