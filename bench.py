@@ -45,7 +45,7 @@ LAUNCHES_PER_STEP = {"c1": 2, "c2": 2, "c3": 2, "c4": 2}
 # from the ncu capture summarised under profiles/ (None until a capture exists).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     "c2": 681.0e6,   # 2 x (336.47 + 4.05) MB: profiles/sparq_decode_pipe_kernel_c2_b32.md (B = 32 capture, scaled by the units)
-    "c3": 540.9e6,   # 510.4 + 30.5 MB: profiles/sparq_decode_pipe_kernel_split_keys_c3.md (the keys' lower halves are written out)
+    "c3": 541.5e6,   # 511.4 + 30.1 MB: profiles/sparq_decode_pipe_kernel_split_keys_c3.md (the keys' lower halves are written out)
     "c4": 812.5e6,   # 808.8 + 3.7 MB: the same file (the heads of a group share rows in the L2)
 }
 

@@ -163,9 +163,9 @@ static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= 
 // The persistent kernel's split-key form against the wide kernel, for caches too long for the persistent
 // kernel's 32-bit keys: with four or more units per SM its hand-built overlap of one unit's stream with
 // the others' select and gather beats the wide kernel's two CTAs per SM (1024 units of 16384 positions
-// at r = 16: 122 against 142 us; 2048 units of 8192 at r = 16: 125 against 156; 1024 units of 8192 at
+// at r = 16: 116 against 142 us; 2048 units of 8192 at r = 16: 125 against 156; 1024 units of 8192 at
 // r = 32: 117 against 132), with fewer it loses (256 units of 16384: 48 against 41).  Beyond about 11,800
-// positions only a 64 KB ring fits beside the keys, which holds the stream back when the rows are many
+// positions only a ring of four or five 16 KB stages fits beside the keys, which holds the stream back when the rows are many
 // (1024 units of 16384 at r = 32: 201 against 195; 512 units at r = 64: 223 against 175): there only up to r = 16.
 static bool pipe16_preferred(int units, int S_max, int r, int n_sm) {
     const int smem = device_info().smem_optin;

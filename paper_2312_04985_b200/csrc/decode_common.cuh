@@ -33,7 +33,6 @@ struct Group {
 
 // What the later stages need to know about one (batch, query head) unit; filled by stage a1.
 struct alignas(16) HeadMeta {
-    float qf[D];                  // q as fp32
     uint16_t q16[D];              // q as stored (fp16 bits)
     int32_t i1[D];                // selected components, ascending
     uint32_t rkey[D];             // a1 scratch: ranking keys
@@ -202,7 +201,7 @@ __device__ __forceinline__ uint32_t group_scan_incl(uint32_t v, uint32_t* red, u
 
 // Stage a1 by a whole CTA (G::NT >= 128 threads): the r largest |q_j| by rank counting.
 // key = |q_j| bit pattern above (127 - j): distinct keys, larger |q| first, then smaller j.
-// Fills hm.qf, q16, i1 (ascending), qh (zero padded to a multiple of RB_), inv_tau, l1_sel.
+// Fills hm.q16, i1 (ascending), qh (zero padded to a multiple of RB_), inv_tau, l1_sel.
 // red: 2*NW floats, cnt: 4 words.  Ends with a barrier.
 template <class G, int RB_>
 __device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restrict__ q_row, int r, HeadMeta& hm, float* red,
@@ -216,7 +215,6 @@ __device__ __forceinline__ void top_r_block(int tid, const sparq_half* __restric
         qf = __half2float(__ushort_as_half(hb));
         aq = fabsf(qf);
         mine = ((uint32_t)(hb & 0x7fffu) << 7) | (uint32_t)(D - 1 - tid);
-        hm.qf[tid] = qf;
         hm.q16[tid] = hb;
         hm.rkey[tid] = mine;
     }
@@ -286,7 +284,7 @@ __device__ __forceinline__ double dot64_at(const sparq_half* Kt_head, const Head
     double acc = 0.0;
     for (int j = 0; j < r; ++j) {
         const int c = hm.i1[j];
-        acc = fma(ldexp((double)hm.qf[c], 1008), h2d_scalar(Kt_head[(size_t)c * S_max + (size_t)t * t_stride]), acc);
+        acc = fma(ldexp((double)__half2float(__ushort_as_half(hm.q16[c])), 1008), h2d_scalar(Kt_head[(size_t)c * S_max + (size_t)t * t_stride]), acc);
     }
     return acc;
 }
@@ -302,7 +300,7 @@ static __device__ __noinline__ double dot64_at_batched(const sparq_half* Kt_head
             kv[u] = j0 + u < r ? Kt_head[(size_t)hm.i1[j0 + u] * S_max + (size_t)t * t_stride] : (uint16_t)0;
 #pragma unroll
         for (int u = 0; u < 16; ++u)
-            if (j0 + u < r) acc = fma(ldexp((double)hm.qf[hm.i1[j0 + u]], 1008), h2d_scalar(kv[u]), acc);
+            if (j0 + u < r) acc = fma(ldexp((double)__half2float(__ushort_as_half(hm.q16[hm.i1[j0 + u]])), 1008), h2d_scalar(kv[u]), acc);
     }
     return acc;
 }

@@ -32,14 +32,19 @@ constexpr int CH = SNT * 8;              // positions per chunk: 8 per stream th
 // measured), or, where the longest caches of the split-key form leave less room, 4 stages of 4 rows (64 KB).
 // Split keys (K16): the keys' upper halves in shared memory, the lower halves in the caller's workspace,
 // where the L2 keeps them; for caches whose 32-bit keys do not fit three times beside the ring.
-template <bool THIN>
+// RING: 0 = 3 x 32 KB, 1 = 4 x 16 KB, 2 = 5 x 16 KB (the split-key form's longest caches, when the budget k is
+// small enough for the fifth stage to fit beside the index lists).
+template <int RING>
 struct Ring {
-    static constexpr int RB = THIN ? 4 : 8;
-    static constexpr int STAGES = THIN ? 4 : 3;
+    static constexpr int RB = RING ? 4 : 8;
+    static constexpr int STAGES = RING == 0 ? 3 : RING == 1 ? 4 : 5;
     static constexpr int STAGE_BYTES = RB * CH * 2;
     static constexpr int BYTES = STAGES * STAGE_BYTES;
 };
-constexpr int STAGES_MAX = 4;
+constexpr int STAGES_MAX = 5;
+// entries of one post group's index list i2 in dynamic shared memory (k rounded up to whole 128-byte lines)
+__host__ __device__ constexpr int i2_pad(int k) { return ((k > 0 ? k : 1) + 31) & ~31; }
+__host__ __device__ constexpr size_t post_scratch_aligned(int S_cap) { return (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127; }
 constexpr int NKB_MAX = 4;               // key buffers: one being written, the others waiting for or in the post groups;
                                          // four where they fit (1.7 us faster on the bench shape), else three
 constexpr int NMETA = 4;                 // unit metadata slots in flight
@@ -61,9 +66,10 @@ __device__ unsigned long long g_pipe_clocks[16];
 #define CLK_ADD(i, var, cond)
 #endif
 
-struct PipeShared {
+template <bool K16>
+struct PipeSharedT {
     HeadMeta meta[NMETA];
-    int32_t i2[NPOST][SPARQ_K_MAX];
+    int32_t i2[NPOST][K16 ? 8 : SPARQ_K_MAX];     // (split keys: the lists live in dynamic shared memory)
     uint64_t full[STAGES_MAX], empty[STAGES_MAX];          // ring stage landed / consumed
     uint64_t meta_full[NMETA], meta_free[NMETA];   // a1 done / unit finished
     uint64_t keys_full[NKB_MAX], keys_free[NKB_MAX];   // keys of a unit complete / post-processed
@@ -107,8 +113,8 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // Bounded wait.  Between polls the warp sleeps NS nanoseconds so that waiting warps leave the issue
 // slots to the working ones.  Gives up after WAIT_LIMIT polls, or at once when another thread
 // already gave up; from then on no wait in this CTA blocks.
-template <int NS>
-__device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, PipeShared& sh, int32_t* status) {
+template <int NS, class SH>
+__device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, SH& sh, int32_t* status) {
     volatile int* flag = &sh.abort_flag;
     for (int i = 0; i < WAIT_LIMIT; ++i) {
         if (mbar_try_wait(bar, parity)) return;
@@ -121,8 +127,8 @@ __device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, Pi
 
 // The same for a whole thread group: its first warp polls, the other warps sleep in the group's
 // hardware barrier instead of spending issue slots on polls.
-template <class G, int NS>
-__device__ __forceinline__ void group_wait(int gtid, uint64_t* bar, uint32_t parity, PipeShared& sh, int32_t* status) {
+template <class G, int NS, class SH>
+__device__ __forceinline__ void group_wait(int gtid, uint64_t* bar, uint32_t parity, SH& sh, int32_t* status) {
     if (gtid < 32) wait_or_abort<NS>(bar, parity, sh, status);
     G::sync();
 }
@@ -141,8 +147,8 @@ __device__ __forceinline__ int next_unit(const Args& a, int bh, int lane) {
     return u < a.n_units ? u : -1;
 }
 
-template <int RB>
-__device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uint32_t opts) {
+template <int RB, class SH>
+__device__ __forceinline__ void a1_role(const Args& a, SH& sh, const uint32_t opts) {
     const int lane = threadIdx.x & 31;
     int bh = (int)blockIdx.x < a.n_units ? (int)blockIdx.x : -1;
     uint2 qraw = make_uint2(0, 0);                           // components 4*lane .. 4*lane+3 of the unit's q
@@ -179,7 +185,6 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uin
             qf[e] = __half2float(__ushort_as_half(hb[e]));
             l1_all += fabsf(qf[e]);
             mine[e] = ((uint32_t)(hb[e] & 0x7fffu) << 7) | (uint32_t)(D - 1 - c);
-            hm.qf[c] = qf[e];
             hm.q16[c] = hb[e];
             hm.rkey[c] = mine[e];
         }
@@ -232,9 +237,9 @@ __device__ __forceinline__ void a1_role(const Args& a, PipeShared& sh, const uin
 }
 
 // ---------------------------------------------------------------------------------- producer
-template <bool THIN>
-__device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, unsigned char* ring, int p) {
-    constexpr int RB = Ring<THIN>::RB, STAGES = Ring<THIN>::STAGES, STAGE_BYTES = Ring<THIN>::STAGE_BYTES;
+template <int RING, class SH>
+__device__ __forceinline__ void producer_role(const Args& a, SH& sh, unsigned char* ring, int p) {
+    constexpr int RB = Ring<RING>::RB, STAGES = Ring<RING>::STAGES, STAGE_BYTES = Ring<RING>::STAGE_BYTES;
     const int lane = threadIdx.x & 31;
     const int g_heads = a.Hq / a.Hkv;
     uint32_t g = 0;                                          // ring stages issued so far
@@ -268,10 +273,10 @@ __device__ __forceinline__ void producer_role(const Args& a, PipeShared& sh, uns
 }
 
 // ---------------------------------------------------------------------------------- stream group
-template <int NKB, bool K16, bool THIN>
-__device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const unsigned char* ring, uint32_t* keys_all,
+template <int NKB, bool K16, int RING, class SH>
+__device__ __forceinline__ void stream_role(const Args& a, SH& sh, const unsigned char* ring, uint32_t* keys_all,
                                             uint32_t* hist1_all) {
-    constexpr int RB = Ring<THIN>::RB, STAGES = Ring<THIN>::STAGES, STAGE_BYTES = Ring<THIN>::STAGE_BYTES;
+    constexpr int RB = Ring<RING>::RB, STAGES = Ring<RING>::STAGES, STAGE_BYTES = Ring<RING>::STAGE_BYTES;
     const int gtid = threadIdx.x - LEAD, lane = gtid & 31;
     int s = 0;                                               // ring slot and its phase parity
     uint32_t parity = 0;
@@ -384,13 +389,13 @@ __device__ __forceinline__ void stream_role(const Args& a, PipeShared& sh, const
 }
 
 // ---------------------------------------------------------------------------------- post groups
-template <class PG, int NKB, bool K16>
-__device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const uint32_t* keys_all, uint32_t* hist1_all,
-                                          unsigned char* scratch, int p, const uint32_t opts) {
+template <class PG, int NKB, bool K16, class SH>
+__device__ __forceinline__ void post_role(const Args& a, SH& sh, const uint32_t* keys_all, uint32_t* hist1_all,
+                                          unsigned char* scratch, int32_t* i2, int p, const uint32_t opts) {
     const int gtid = threadIdx.x - LEAD - SNT - p * GNT;
     PostScratch sc;
     carve_post_scratch(sc, scratch, PG::NHW, a.S_cap / 32);
-    sc.i2 = sh.i2[p]; sc.red = sh.red[p]; sc.redu = sh.redu[p]; sc.res = sh.res[p]; sc.band = sh.band[p];
+    sc.i2 = i2; sc.red = sh.red[p]; sc.redu = sh.redu[p]; sc.res = sh.res[p]; sc.band = sh.band[p];
     const int g_heads = a.Hq / a.Hkv;
     for (int j = p;; j += NPOST) {
         const int m = j % NMETA, kb = j % NKB;
@@ -454,17 +459,20 @@ __device__ __forceinline__ void post_role(const Args& a, PipeShared& sh, const u
 
 // OPT = false: the paper's algorithm as stated, the settings word known to be 0 at compile time (the
 // instantiation the plain decode call runs); OPT = true: settings taken from `opts_arg`.
-template <int NKB, bool OPT, bool K16, bool THIN>
+template <int NKB, bool OPT, bool K16, int RING>
 __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, const uint32_t opts_arg) {
-    using R = Ring<THIN>;
+    using R = Ring<RING>;
     const uint32_t opts = OPT ? opts_arg : 0u;
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     unsigned char* ring = dyn_smem;
     uint32_t* keys_all = reinterpret_cast<uint32_t*>(dyn_smem + R::BYTES);     // NKB buffers of S_cap keys (split keys: their upper halves)
     uint32_t* hist1_all = keys_all + (size_t)NKB * a.S_cap / (K16 ? 2 : 1);   // per key buffer: histogram of the keys' top bits
     unsigned char* scratch0 = reinterpret_cast<unsigned char*>(hist1_all + NKB * FBINS);
-    const size_t scratch_bytes = (post_scratch_bytes(GNT / 16, a.S_cap / 32) + 127) & ~(size_t)127;
-    __shared__ PipeShared sh;
+    const size_t scratch_bytes = post_scratch_aligned(a.S_cap);
+    // the post groups' index lists: SPARQ_K_MAX entries each in static shared memory, or, with split keys (whose
+    // longest caches need the room), i2_pad(k) entries each behind the scratch areas
+    int32_t* i2_dyn = reinterpret_cast<int32_t*>(scratch0 + NPOST * scratch_bytes);
+    __shared__ PipeSharedT<K16> sh;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < R::STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], SNT / 32); }
@@ -479,17 +487,18 @@ __global__ void __launch_bounds__(NT, 1) sparq_decode_pipe_kernel(const Args a, 
     if (threadIdx.x == 0) { unsigned long long gt; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt)); g_cta_begin[blockIdx.x] = gt; g_cta_end[blockIdx.x] = 0; }
 #endif
     const int warp = threadIdx.x >> 5;
-    if (warp < NPROD) producer_role<THIN>(a, sh, ring, warp);
+    if (warp < NPROD) producer_role<RING>(a, sh, ring, warp);
     else if (warp == NPROD) a1_role<R::RB>(a, sh, opts);
-    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB, K16, THIN>(a, sh, ring, keys_all, hist1_all);
-    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB, K16>(a, sh, keys_all, hist1_all, scratch0, 0, opts);
-    else post_role<PG1, NKB, K16>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, 1, opts);
+    else if (warp < LEAD / 32 + SNT / 32) stream_role<NKB, K16, RING>(a, sh, ring, keys_all, hist1_all);
+    else if (warp < LEAD / 32 + SNT / 32 + GNT / 32) post_role<PG0, NKB, K16>(a, sh, keys_all, hist1_all, scratch0, K16 ? i2_dyn : sh.i2[0], 0, opts);
+    else post_role<PG1, NKB, K16>(a, sh, keys_all, hist1_all, scratch0 + scratch_bytes, K16 ? i2_dyn + i2_pad(a.k) : sh.i2[1], 1, opts);
 }
 
-size_t pipe_dynamic_smem(int S_cap, int NKB, bool k16, bool thin) {
-    const size_t scratch = (post_scratch_bytes(GNT / 16, S_cap / 32) + 127) & ~(size_t)127;
-    return (size_t)(thin ? Ring<true>::BYTES : Ring<false>::BYTES) + (size_t)NKB * S_cap * (k16 ? 2 : 4) +
-           (size_t)NKB * FBINS * 4 + NPOST * scratch;
+size_t pipe_dynamic_smem(int S_cap, int NKB, bool k16, int ring, int k) {
+    const size_t scratch = post_scratch_aligned(S_cap);
+    const size_t ring_bytes = ring == 0 ? Ring<0>::BYTES : ring == 1 ? Ring<1>::BYTES : Ring<2>::BYTES;
+    return ring_bytes + (size_t)NKB * S_cap * (k16 ? 2 : 4) + (size_t)NKB * FBINS * 4 + NPOST * scratch +
+           (k16 ? (size_t)NPOST * i2_pad(k) * 4 : 0);
 }
 constexpr int NKB_SPLIT = 3;             // key buffers of the split-key form
 
@@ -519,12 +528,13 @@ extern "C" int sparq_debug_post_clocks(unsigned long long* out16, int reset) {
 // S_max rounded up so that bitmap words and 16-byte key vectors stay whole
 static int pipe_s_cap(int S_max) { return (S_max + 127) & ~127; }
 
-static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb, bool k16, bool thin) {
-    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb, k16, thin) + sizeof(PipeShared) + 1024 <= (size_t)smem_optin;
+// (the plan selection asks without knowing k: the largest budget's index lists are assumed)
+static bool pipe_fits_nkb(int S_max, int smem_optin, int nkb, bool k16, int ring, int k = SPARQ_K_MAX) {
+    return pipe_dynamic_smem(pipe_s_cap(S_max), nkb, k16, ring, k) + (k16 ? sizeof(PipeSharedT<true>) : sizeof(PipeSharedT<false>)) + 1024 <= (size_t)smem_optin;
 }
-bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3, false, false); }
-bool pipe_split_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, true); }
-bool pipe_split_thin_ring(int S_max, int smem_optin) { return !pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, false); }
+bool pipe_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, 3, false, 0); }
+bool pipe_split_fits(int S_max, int smem_optin) { return pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, 1); }
+bool pipe_split_thin_ring(int S_max, int smem_optin) { return !pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, 0); }
 // Workspace of the split-key form: the unit counter, then the keys' lower halves.
 size_t pipe_split_workspace(int S_max, int n_sm) { return SPLIT_LO_OFFSET + (size_t)n_sm * NKB_SPLIT * pipe_s_cap(S_max) * 2; }
 
@@ -540,13 +550,16 @@ cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, c
     a.out = out; a.idx_r = idx_r; a.idx_k = idx_k; a.alpha = alpha; a.status = status; a.unit_counter = unit_counter;
     const int smem_optin = device_info().smem_optin;
     const bool k16 = split_keys && unit_counter;
-    const bool four = !k16 && pipe_fits_nkb(S_max, smem_optin, 4, false, false);
-    const bool thin = k16 && pipe_split_thin_ring(S_max, smem_optin);
-    const size_t dyn = pipe_dynamic_smem(a.S_cap, k16 ? NKB_SPLIT : (four ? 4 : 3), k16, thin);
-    auto kernel = k16 ? (thin ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, true> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, true>)
-                              : (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, false> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, false>))
-                : opts ? (four ? sparq_decode_pipe_kernel<4, true, false, false> : sparq_decode_pipe_kernel<3, true, false, false>)
-                       : (four ? sparq_decode_pipe_kernel<4, false, false, false> : sparq_decode_pipe_kernel<3, false, false, false>);
+    const bool four = !k16 && pipe_fits_nkb(S_max, smem_optin, 4, false, 0);
+    // split keys: the 96 KB ring where it fits whatever the budget; else five 16 KB stages if this call's k leaves room, else four
+    const int ring = !k16 ? 0 : pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, 0) ? 0
+                                : pipe_fits_nkb(S_max, smem_optin, NKB_SPLIT, true, 2, k) ? 2 : 1;
+    const size_t dyn = pipe_dynamic_smem(a.S_cap, k16 ? NKB_SPLIT : (four ? 4 : 3), k16, ring, k);
+    auto kernel = k16 ? (ring == 0 ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, 0> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, 0>)
+                       : ring == 1 ? (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, 1> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, 1>)
+                                   : (opts ? sparq_decode_pipe_kernel<NKB_SPLIT, true, true, 2> : sparq_decode_pipe_kernel<NKB_SPLIT, false, true, 2>))
+                : opts ? (four ? sparq_decode_pipe_kernel<4, true, false, 0> : sparq_decode_pipe_kernel<3, true, false, 0>)
+                       : (four ? sparq_decode_pipe_kernel<4, false, false, 0> : sparq_decode_pipe_kernel<3, false, false, 0>);
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
     if (e != cudaSuccess) return e;
     const int grid = a.n_units < n_sm ? a.n_units : n_sm;
