@@ -133,7 +133,7 @@ int sparq_cache_append(const sparq_half* k_new, const sparq_half* v_new,
  * of a unit pass through the workspace (4 bytes per position), and with few units every sequence
  * is cut into slices handled by different thread blocks; more units than SMs on the persistent
  * kernel -- 64 bytes for a counter from which the thread blocks draw their units, which evens
- * out their finishing times; four or more units per SM on a cache of about 6,000 to 17,000
+ * out their finishing times; four or more units per SM on a cache of about 6,500 to 17,800
  * positions -- the persistent kernel keeps only the upper halves of the scores' sort keys in
  * shared memory and parks the lower halves here (SMs x 3 x 2 bytes per position).  With
  * workspace NULL or too small a plan without scratch is used.  The call clears what it needs;

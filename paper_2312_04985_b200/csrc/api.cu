@@ -47,7 +47,7 @@ int device_sm_count() { return device_info().sm_count; }
 // Unset or anything else: the wide kernel (one CTA of 512 threads, or two of 256, per SM; a unit's
 // keys in shared memory) for up to two units per SM and for caches too long for the persistent
 // kernel; the persistent pipelined kernel wherever else one unit's keys fit its shared memory, and in
-// its split-key form (pipe16) for four or more units per SM on caches up to about 17,000 positions;
+// its split-key form (pipe16) for four or more units per SM on caches up to about 17,800 positions;
 // beyond the wide kernel's reach (about 44,000 positions) the split plan if the caller passed its
 // workspace; else one CTA per unit.
 int forced_plan() {
@@ -164,7 +164,7 @@ static bool wide_preferred(int units, int n_sm, bool pipe_ok) { return units <= 
 // kernel's 32-bit keys: with four or more units per SM its hand-built overlap of one unit's stream with
 // the others' select and gather beats the wide kernel's two CTAs per SM (1024 units of 16384 positions
 // at r = 16: 116 against 142 us; 2048 units of 8192 at r = 16: 125 against 156; 1024 units of 8192 at
-// r = 32: 117 against 132), with fewer it loses (256 units of 16384: 48 against 41).  Beyond about 11,800
+// r = 32: 117 against 132), with fewer it loses (256 units of 16384: 48 against 41).  Beyond about 12,700
 // positions only a ring of four or five 16 KB stages fits beside the keys, which holds the stream back when the rows are many
 // (1024 units of 16384 at r = 32: 201 against 195; 512 units at r = 64: 223 against 175): there only up to r = 16.
 static bool pipe16_preferred(int units, int S_max, int r, int n_sm) {

@@ -44,7 +44,7 @@ cudaError_t launch_sparq_decode_split(const sparq_half* q, const sparq_half* K, 
 // bytes of the caller's workspace): reaches caches about three times as long.
 bool pipe_fits(int S_max, int smem_optin);
 bool pipe_split_fits(int S_max, int smem_optin);
-bool pipe_split_thin_ring(int S_max, int smem_optin);    // only a ring of 16 KB stages fits beside the keys (S_max beyond about 11,800)
+bool pipe_split_thin_ring(int S_max, int smem_optin);    // only a ring of 16 KB stages fits beside the keys (S_max beyond about 12,700)
 size_t pipe_split_workspace(int S_max, int n_sm);
 cudaError_t launch_sparq_decode_pipe(const sparq_half* q, const sparq_half* K, const sparq_half* Kt, const sparq_half* V,
                                      const sparq_half* vbar, const int32_t* seq_lens, int B, int Hq, int Hkv, int S_max,
